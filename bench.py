@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the AWE exact integer matrix product on B200.
+
+One "step" is one pass of the whole hot path over one batch: encode A, encode B, the r FP4
+GEMMs with the fused integer reconstruction.  The default workload is the one the headline
+metric is quoted on: INT8 x INT8 at M = N = K = 8192 with the 6-product encoding.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is effective exact-INT8 TOPS = 2 M N K / t with inputs
+resident in HBM; `e2e` is the same metric through awe_gemm_exact_host with pinned HOST buffers
+(host<->device copies inside the timed region); `roofline` describes the dominant kernel (the
+FP4 GEMM) against the FP4 tensor peak; `cpu_baseline` is the CPU oracle timed on a bounded
+sample of the same workload on this machine's cores.  With --gpus N > 1 (under torchrun) every
+rank runs an independent replica of the workload: the path has no exchange step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "effective exact INT8xINT8 TOPS (2*M*N*K / time), AWE 6-GEMM"
+NOMINAL_FP4_TFLOPS = 9000.0          # published dense FP4 peak of one B200 (paper, Section 6.2)
+NOMINAL_FP4_OVER_BF16 = 4.0          # 9.0 / 2.25 PFLOP/s nominal
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed regions run."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting"}
+
+    def __init__(self, index: int, uuid: str = ""):
+        self.samples, self.reasons, self.max_mhz, self.power = [], set(), None, []
+        self._stop = threading.Event()
+        self._active = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:
+                self._dev = pynvml.nvmlDeviceGetHandleByUUID(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+            except Exception:
+                self._dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._dev, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            if self._active.is_set():
+                try:
+                    self.samples.append(nv.nvmlDeviceGetClockInfo(self._dev, nv.NVML_CLOCK_SM))
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._dev)
+                    for bit, name in self.REASONS.items():
+                        if mask & bit:
+                            self.reasons.add(name)
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(self._dev) / 1000.0)
+                except Exception:
+                    pass
+            time.sleep(0.005)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def region(self, on: bool):
+        (self._active.set if on else self._active.clear)()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": max(self.power) if self.power else None}
+
+
+def cpu_oracle_sample(A, B, budget_s: float):
+    """Time the CPU oracle (plain int64 product) on the first rows of the workload; the number
+    of rows is chosen from a 2-row probe so the run takes about budget_s seconds."""
+    from oracle import matmul as om
+    om.build()
+    M, K = A.shape
+    N = B.shape[1]
+    t0 = time.perf_counter()
+    om.matmul_i64_rows(A, B, 0, min(2 * om.threads(), M))
+    probe = (time.perf_counter() - t0) / min(2 * om.threads(), M)
+    rows = int(max(om.threads(), min(M, budget_s / max(probe, 1e-9))))
+    t0 = time.perf_counter()
+    om.matmul_i64_rows(A, B, 0, rows)
+    dt = time.perf_counter() - t0
+    return {"value": 2.0 * rows * N * K / dt / 1e12, "unit": "TOPS", "cores": om.threads(), "kind": "oracle",
+            "sample": f"rows 0..{rows - 1} of the {M}x{N}x{K} product ({dt:.1f} s)"}, rows, dt
+
+
+def run_reference(args, w, rank):
+    """The reference arm is the CPU oracle as it stands, on this machine's cores."""
+    if rank != 0:
+        return
+    from paper_2609_24519_b200 import workloads as wl
+    from oracle import matmul as om
+    om.build()
+    A, B = wl.make_inputs(w)
+    per_step = max(0.3, min(3.0, 150.0 / max(1, args.steps + args.warmup)))
+    _, rows, dt = cpu_oracle_sample(A, B, per_step)
+    for _ in range(args.warmup):
+        om.matmul_i64_rows(A, B, 0, rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        om.matmul_i64_rows(A, B, 0, rows)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = 2.0 * rows * w.N * w.K / dt / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K,
+                       "note": "CPU oracle; each step is a bounded row sample of the workload"},
+            "cpu_baseline": {"value": value, "unit": "TOPS", "cores": om.threads(), "kind": "oracle",
+                             "sample": f"rows 0..{rows - 1} of {w.M} per step"},
+            "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--size", type=int, default=8192, help="M = N = K of the headline workload")
+    ap.add_argument("--no-extras", action="store_true", help="skip the context measurements")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2609_24519_b200 import workloads as wl
+    w = wl.headline(args.size)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, w, rank)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_24519_b200 import binding as b
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    h = b.awe_create(local_rank)
+    enc, M, N, K = b.ENC_INT8_AWE6, w.M, w.N, w.K
+    A, B = wl.make_inputs(w)
+    dA, dB = torch.from_numpy(A).to(dev), torch.from_numpy(B).to(dev)
+    C = torch.empty((M, N), dtype=torch.int32, device=dev)
+    nA = b.awe_planes_bytes(enc, 0, b.SIDE_A, M, K)
+    ws = torch.empty(b.awe_workspace_bytes(enc, 0, M, N, K), dtype=torch.uint8, device=dev)
+    pa, pb = ws[:nA], ws[(nA + 255) // 256 * 256:]
+    desc = b.awe_encoding_info(enc)
+
+    def step(events=None):
+        if events is not None:
+            events[0].record()
+        b.awe_encode(h, enc, 0, b.SIDE_A, dA, b.I8, b.ROWMAJOR_RxK, M, K, K, pa)
+        b.awe_encode(h, enc, 0, b.SIDE_B, dB, b.I8, b.ROWMAJOR_KxR, N, K, N, pb)
+        if events is not None:
+            events[1].record()
+        b.awe_gemm_planes(h, enc, 0, pa, pb, M, N, K, C, b.C_I32, N)
+        if events is not None:
+            events[2].record()
+
+    # ---- parity on sampled rows (outside every timed region)
+    from oracle import matmul as om
+    om.build()
+    step()
+    torch.cuda.synchronize()
+    rows = sorted(set(np.random.default_rng(0).integers(0, M, 8).tolist() + [0, M - 1]))
+    got = C[rows].cpu().numpy().astype(np.int64)
+    parity_ok = all(np.array_equal(got[i], om.matmul_i64_rows(A, B, r, r + 1)[0]) for i, r in enumerate(rows))
+    # the single-call entry point must give the same matrix as the three calls
+    C2 = torch.empty_like(C)
+    b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, enc, 0, C2, b.C_I32, ws)
+    torch.cuda.synchronize()
+    parity_ok = parity_ok and bool(torch.equal(C, C2)) and b.awe_last_device_status(h) == (0, 0)
+
+    sampler = ClockSampler(local_rank, str(getattr(torch.cuda.get_device_properties(dev), "uuid", "")))
+    sampler.start()
+
+    # ---- device-resident timing
+    for _ in range(args.warmup):
+        step()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = b.awe_launch_count(h)
+    barrier()
+    sampler.region(True)
+    t_start.record()
+    for i in range(args.steps):
+        step(evs[i])
+    t_end.record()
+    barrier()
+    sampler.region(False)
+    launches = b.awe_launch_count(h) - launches0
+    ms_total = t_start.elapsed_time(t_end)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    ms_encode = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+    ms_gemm = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    assert b.awe_last_device_status(h) == (0, 0)
+
+    # ---- end to end from pinned host buffers through awe_gemm_exact_host
+    Ah, Bh = torch.from_numpy(A).pin_memory(), torch.from_numpy(B).pin_memory()
+    Ch = torch.empty((M, N), dtype=torch.int32).pin_memory()
+    scratch = torch.empty(b.awe_workspace_bytes(enc, 0, M, N, K) + b.awe_host_staging_bytes(enc, 0, M, N, K, b.C_I32),
+                          dtype=torch.uint8, device=dev)
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        b.awe_gemm_exact_host(h, Ah, b.I8, Bh, b.I8, M, N, K, enc, 0, Ch, b.C_I32, scratch)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.region(True)
+    e0.record()
+    for _ in range(e2e_steps):
+        b.awe_gemm_exact_host(h, Ah, b.I8, Bh, b.I8, M, N, K, enc, 0, Ch, b.C_I32, scratch)
+    e1.record()
+    barrier()
+    sampler.region(False)
+    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    parity_ok = parity_ok and bool(torch.equal(Ch, C.cpu()))
+    clocks = sampler.stop()
+
+    ops = 2.0 * M * N * K
+    peaks = measured_peaks()
+    fp4_peak = peaks["bf16_tflops_sustained"] * NOMINAL_FP4_OVER_BF16
+    gemm_tflops = desc.r * ops / (ms_gemm * 1e-3) / 1e12
+    line = {
+        "metric": METRIC, "value": world * ops / (ms_step * 1e-3) / 1e12, "unit": "TOPS", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "e2m1 (fp4) operands, f32 accumulate, int32 reconstruction",
+        "data": "synthetic",
+        "config": {"workload": w.name, "M": M, "N": N, "K": K, "encoding": "int8_awe6", "fp4_gemms": desc.r,
+                   "inputs": "int8 uniform [-128,127], numpy default_rng(seed=6)", "output": "int32",
+                   "l2": "no flush: per-step working set (64+64 MiB in, 384 MiB planes, 256 MiB out) exceeds the 126 MB L2",
+                   "parallelism": "replicas only (no exchange step)" if world > 1 else "single GPU"},
+        "clocks": clocks,
+        "e2e": {"value": world * ops / (ms_e2e * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms_e2e,
+                "steps": e2e_steps, "h2d_bytes_per_step": int(A.nbytes + B.nbytes), "d2h_bytes_per_step": int(M * N * 4)},
+        "gpu_launches": int(launches),
+        "parity": "bit-exact vs CPU oracle on %d sampled rows; 3-call path == awe_gemm_exact == host path" % len(rows)
+                  if parity_ok else "MISMATCH",
+        "kernels_ms": {"encode_a_plus_b": ms_encode, "gemm_and_reconstruction": ms_gemm},
+        "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
+                     "frac": gemm_tflops / fp4_peak, "traffic": None,
+                     "kernel": "awe_gemm_kernel", "flops_per_launch": desc.r * ops,
+                     "peak_source": "%s bf16 sustained %.1f TFLOP/s x nominal fp4:bf16 ratio 4" %
+                                    (peaks["source"], peaks["bf16_tflops_sustained"]),
+                     "frac_of_nominal_9pflops": gemm_tflops / NOMINAL_FP4_TFLOPS,
+                     "frac_of_burst_peak": gemm_tflops / (peaks["bf16_tflops"] * NOMINAL_FP4_OVER_BF16)},
+        "encode_roofline": {"bound": "hbm", "achieved": (M * K + K * N) * (1 + desc.n_planes_a / 2.0) / (ms_encode * 1e-3) / 1e9,
+                            "peak": peaks["hbm_gbs"], "unit": "GB/s"},
+    }
+    line["encode_roofline"]["frac"] = line["encode_roofline"]["achieved"] / peaks["hbm_gbs"]
+
+    if rank == 0 and not args.no_extras:
+        ctx = {}
+        # prior-work 9-GEMM base-13 scheme through the same kernels, same inputs
+        enc9 = b.ENC_INT8_BASE13_9
+        ws9 = torch.empty(b.awe_workspace_bytes(enc9, 0, M, N, K), dtype=torch.uint8, device=dev)
+        C9 = torch.empty_like(C)
+        for _ in range(2):
+            b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, enc9, 0, C9, b.C_I32, ws9)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(5):
+            b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, enc9, 0, C9, b.C_I32, ws9)
+        e1.record()
+        torch.cuda.synchronize()
+        ctx["base13_9gemm_TOPS"] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
+        ctx["base13_equals_awe6"] = bool(torch.equal(C9, C))
+        del ws9, C9
+        # INT8 tensor-core GEMM of the same product (library reference point)
+        try:
+            for _ in range(2):
+                Ci = torch._int_mm(dA, dB)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(5):
+                Ci = torch._int_mm(dA, dB)
+            e1.record()
+            torch.cuda.synchronize()
+            ctx["int8_tensor_core_gemm_TOPS"] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
+            ctx["int8_gemm_equals_awe6"] = bool(torch.equal(Ci, C))
+            del Ci
+        except Exception as ex:  # library reference point only
+            ctx["int8_tensor_core_gemm_TOPS"] = None
+            ctx["int8_gemm_error"] = str(ex)[:100]
+        ctx["paper_theoretical_TOPS"] = "1500 (9.0 PFLOPS / 6, published peak, not a measurement; B200)"
+        line["context"] = ctx
+
+    if rank == 0 and world == 1 and not args.no_cpu:
+        line["cpu_baseline"] = cpu_oracle_sample(A, B, 12.0)[0]
+    elif rank == 0:
+        line["cpu_baseline"] = None
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,183 @@
+/* awe.h -- C ABI of the B200 (sm_100a) library for error-free integer matrix products
+ * computed as a few FP4 (E2M1) tensor-core GEMMs under Adaptive Weight Encoding (AWE).
+ *
+ * What the library computes is the run-time procedure of the paper (Algorithm 1):
+ *   1. every entry of A and of B is decomposed into limbs by table lookup and the stored
+ *      planes (linear combinations of limbs, every value in S = {0,+-1,+-2,+-3,+-4,+-6,+-8,+-12})
+ *      are written as packed E2M1 (awe_encode);
+ *   2. for each product k = 1..r, P_k = plane alpha_k of A times plane beta_k of B on the FP4
+ *      tensor cores with FP32 accumulation, the reduction dimension cut into segments short
+ *      enough (Section 3.4, K*) that every partial sum is an integer below 2^24 and exact;
+ *   3. C = (sum_k l_k P_k) / D in integers, D a power of two (Definition 4.1), or the same sum
+ *      reduced mod m for the residue form (Section 5.3)
+ *   (steps 2 and 3: awe_gemm_planes; all three: awe_gemm_exact).
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise:
+ *   - Pointers named *_dev are DEVICE pointers into memory the caller owns (cudaMalloc'd or a
+ *     framework tensor); pointers named *_host are HOST pointers.  The library never frees or
+ *     keeps a caller pointer past the call's enqueued work.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Device
+ *     work is enqueued on it and the call returns without waiting, except where stated.
+ *   - No entry point allocates device memory per call; scratch is caller-provided
+ *     (awe_workspace_bytes).  A handle owns a small device status word and the encode tables.
+ *   - Errors the host can see (bad argument, unsupported encoding, misalignment, short
+ *     workspace, result range) are returned before anything is enqueued.  Conditions only the
+ *     device can see (a bounded wait inside a kernel ran out) are recorded in the handle's
+ *     status word and reported by awe_last_device_status.
+ *   - There is no CPU fallback: without a CUDA device awe_create fails with AWE_ERR_CUDA.
+ *   - One handle serves one device; calls on one handle must not run concurrently from
+ *     several host threads.
+ */
+#ifndef AWE_H_
+#define AWE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct awe_ctx* awe_handle_t;
+
+typedef enum {
+    AWE_OK = 0,
+    AWE_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, unknown enum value            */
+    AWE_ERR_UNSUPPORTED = 2, /* encoding/modulus/dtype combination the library does not have   */
+    AWE_ERR_WORKSPACE = 3,   /* caller-provided scratch is too small                           */
+    AWE_ERR_ALIGNMENT = 4,   /* a pointer or leading dimension misses its alignment            */
+    AWE_ERR_RANGE = 5,       /* the exact result cannot fit the requested output type          */
+    AWE_ERR_CUDA = 6,        /* a CUDA runtime or driver call failed                           */
+    AWE_ERR_TIMEOUT = 7      /* a bounded wait inside a kernel expired (device status word)    */
+} awe_status_t;
+
+/* Encodings (configuration records of Algorithm 1). */
+typedef enum {
+    AWE_ENC_INT8_AWE6 = 1,      /* INT8xINT8, 6 products, w = v = (1,29,37)   (Section 4.3, Appendix A) */
+    AWE_ENC_INT8_BASE13_9 = 2,  /* INT8xINT8, 9 products, weights (1,13,169)  (prior work, Section 1)  */
+    AWE_ENC_INT4xINT8_AWE4 = 3, /* INT4xINT8, 4 products, D = 2               (Appendix A)             */
+    AWE_ENC_MOD_M = 4,          /* residue form mod `modulus`, 1/3/4 products (Section 5.3)            */
+    AWE_ENC_INT8_AWE6_ALT = 5   /* INT8xINT8, 6 products, w = v = (1,11,39)   (Section 4.3)            */
+} awe_encoding_t;
+
+typedef enum {
+    AWE_I8 = 0,      /* one signed 8-bit value per byte                                          */
+    AWE_I4_IN_I8 = 1 /* one signed 4-bit value per byte; only the low nibble is read (sign-extended) */
+} awe_in_dtype_t;
+
+typedef enum {
+    AWE_C_I32 = 0,     /* exact product, int32 (rejected with AWE_ERR_RANGE if it might not fit) */
+    AWE_C_I64 = 1,     /* exact product, int64                                                   */
+    AWE_C_RES_I16 = 2, /* residue in [-floor(m/2), ceil(m/2)-1], int16 (AWE_ENC_MOD_M only)      */
+    AWE_C_RES_I32 = 3  /* same residue, int32                                                    */
+} awe_out_dtype_t;
+
+typedef enum { AWE_SIDE_A = 0, AWE_SIDE_B = 1 } awe_side_t;
+
+/* How the operand handed to awe_encode is laid out.  R is M for side A and N for side B. */
+typedef enum {
+    AWE_ROWMAJOR_RxK = 0, /* element (row r, reduction index k) at X[r*ld + k]  (A as M x K)     */
+    AWE_ROWMAJOR_KxR = 1  /* element (r, k) at X[k*ld + r]                      (B as K x N)     */
+} awe_layout_t;
+
+#define AWE_MAX_PRODUCTS 16
+#define AWE_MAX_PLANES 8
+
+/* Host-side description of one configuration record (Definition 4.1 / Algorithm 1). */
+typedef struct {
+    int32_t r;                      /* number of products = number of FP4 GEMMs                  */
+    int32_t n_planes_a, n_planes_b; /* distinct stored planes per side                           */
+    int32_t ia[AWE_MAX_PRODUCTS];   /* product k multiplies stored plane ia[k] of A ...          */
+    int32_t ib[AWE_MAX_PRODUCTS];   /* ... by stored plane ib[k] of B                            */
+    int32_t ell[AWE_MAX_PRODUCTS];  /* integer reconstruction coefficients l_k                   */
+    int32_t log2D;                  /* C = (sum l_k P_k) >> log2D                                */
+    int32_t modulus;                /* 0 for the exact encodings                                 */
+    int32_t c_a, c_b;               /* largest |stored plane value| per side (Section 3.4)       */
+    int64_t k_star;                 /* floor(2^24 / (c_a c_b))                                   */
+    int32_t a_lo, a_hi, b_lo, b_hi; /* input value range each side's table covers                */
+} awe_encoding_desc;
+
+/* Create / destroy a handle bound to CUDA device `device`.  awe_create makes that device
+ * current, allocates the handle's status word and table arena (a few hundred KB, once) and
+ * fails with AWE_ERR_CUDA if there is no usable sm_100 device.  (No counterpart in the paper.) */
+awe_status_t awe_create(awe_handle_t* out, int device);
+awe_status_t awe_destroy(awe_handle_t h);
+
+/* Configuration record of an encoding (Definition 4.1; Appendix A; Section 5.3 for MOD_M, where
+ * `modulus` in [2,169] selects the scheme and must be 0 otherwise).  Host only, needs no GPU.
+ * AWE_ERR_UNSUPPORTED if no scheme exists for the modulus. */
+awe_status_t awe_encoding_info(int enc, int modulus, awe_encoding_desc* out);
+
+/* Decomposition table of one side (first two loops of Algorithm 1), host only: for every
+ * raw input byte b (index b & 0xFF, interpreted per `dt`) the n_planes stored plane values,
+ * lut_host[256 * n_planes], row b.  Used to compare the table against an independent one. */
+awe_status_t awe_encoding_lut(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, int8_t* lut_host);
+
+/* Bytes of the packed-plane buffer of one operand: n_planes x R x pitch, pitch =
+ * round_up(K,256)/2 bytes (E2M1, two values per byte, even k in the low nibble, zero padded
+ * along K).  0 on invalid arguments. */
+size_t awe_planes_bytes(int enc, int modulus, awe_side_t side, int64_t R, int64_t K);
+
+/* Bytes of scratch awe_gemm_exact needs (planes of A, then planes of B, each 256-B aligned). */
+size_t awe_workspace_bytes(int enc, int modulus, int64_t M, int64_t N, int64_t K);
+
+/* Extra device scratch awe_gemm_exact_host needs in addition to awe_workspace_bytes: room for
+ * device copies of A, B and C. */
+size_t awe_host_staging_bytes(int enc, int modulus, int64_t M, int64_t N, int64_t K, awe_out_dtype_t out_dt);
+
+/* Encode one operand (Algorithm 1, first two loops): table lookup per value, plane formation,
+ * E2M1 packing.  X_dev: R x K integers laid out per `layout` with leading dimension ld (elements).
+ * planes_dev: awe_planes_bytes bytes, 256-B aligned.  Any ld and any alignment of X_dev are accepted
+ * (16-B aligned X_dev and ld % 16 == 0 take the vectorised path). */
+awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_side_t side, const void* X_dev,
+                        awe_in_dtype_t dt, awe_layout_t layout, int64_t R, int64_t K, int64_t ld,
+                        void* planes_dev, void* stream);
+
+/* Products and reconstruction (Algorithm 1, third loop and last step; Section 3.4 for the
+ * segmentation of K; Section 5.3 for the residue form) on planes written by awe_encode.
+ * C_dev: M x N row-major with leading dimension ldc (elements of the output type), aligned to its
+ * element size (16-B aligned rows, i.e. C_dev % 16 == 0 and ldc*sizeof(elem) % 16 == 0, take
+ * the vector-store path).  k_chunk = 0 lets the library choose the segment length
+ * (<= K* and a multiple of 256); a positive multiple of 256 forces it (testing). */
+awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, const void* planesA_dev,
+                             const void* planesB_dev, int64_t M, int64_t N, int64_t K, void* C_dev,
+                             awe_out_dtype_t out_dt, int64_t ldc, int64_t k_chunk, void* stream);
+
+/* The whole of Algorithm 1: C = A.B exactly (or C mod m).  A_dev: M x K row-major (ld = K),
+ * B_dev: K x N row-major (ld = N), C_dev: M x N row-major (ld = N).  workspace_dev: at least
+ * awe_workspace_bytes bytes, 256-B aligned; its contents are overwritten. */
+awe_status_t awe_gemm_exact(awe_handle_t h, const void* A_dev, awe_in_dtype_t a_dt, const void* B_dev,
+                            awe_in_dtype_t b_dt, int64_t M, int64_t N, int64_t K, int enc, int modulus,
+                            void* C_dev, awe_out_dtype_t out_dt, void* workspace_dev, size_t workspace_bytes,
+                            void* stream);
+
+/* Same product with HOST operands and result: copies A_host and B_host to the device, runs
+ * awe_gemm_exact, copies C back to C_host and waits for the stream, so C_host is valid on return.
+ * scratch_dev must hold awe_workspace_bytes + awe_host_staging_bytes bytes (256-B aligned).
+ * Pinned host memory makes the copies asynchronous with respect to other streams. */
+awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, awe_in_dtype_t a_dt, const void* B_host,
+                                 awe_in_dtype_t b_dt, int64_t M, int64_t N, int64_t K, int enc, int modulus,
+                                 void* C_host, awe_out_dtype_t out_dt, void* scratch_dev, size_t scratch_bytes,
+                                 void* stream);
+
+/* One raw FP4 product P = X.Y^T with FP32 accumulation over all of K in a single segment
+ * (Algorithm 1's "FP4-GEMM" alone; Section 3.4 is the claim this lets a test probe).
+ * planeX_dev: M x pitch bytes, planeY_dev: N x pitch bytes, pitch = round_up(K,256)/2, packed E2M1;
+ * P_dev: M x N float, leading dimension ldp.  The values returned are in the doubled-integer
+ * convention of Section 3.1 (each operand counted as an element of S). */
+awe_status_t awe_fp4_product_raw(awe_handle_t h, const void* planeX_dev, const void* planeY_dev, int64_t M,
+                                 int64_t N, int64_t K, float* P_dev, int64_t ldp, void* stream);
+
+/* Wait for `stream` and read the handle's device status word: AWE_OK, or AWE_ERR_TIMEOUT with
+ * *site (may be NULL) naming the wait that gave up.  The word is cleared by the read. */
+awe_status_t awe_last_device_status(awe_handle_t h, void* stream, int* site);
+
+/* Number of this library's kernels launched through the handle since it was created. */
+int64_t awe_launch_count(awe_handle_t h);
+
+const char* awe_status_string(awe_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AWE_H_ */

@@ -1,0 +1,152 @@
+// Handle management and the whole-procedure entry points (Algorithm 1 end to end).
+#include <cstring>
+#include <new>
+
+#include "awe_internal.h"
+
+using namespace awe;
+
+extern "C" awe_status_t awe_create(awe_handle_t* out, int device) {
+    if (!out) return AWE_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return AWE_ERR_CUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return AWE_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return AWE_ERR_CUDA;
+    if (prop.major != 10) return AWE_ERR_CUDA;  // the kernels are built for sm_100a only
+    awe_ctx* h = new (std::nothrow) awe_ctx();
+    if (!h) return AWE_ERR_CUDA;
+    h->device = device;
+    h->sm_count = prop.multiProcessorCount;
+    if (cudaMalloc(&h->status_dev, 2 * sizeof(unsigned int)) != cudaSuccess ||
+        cudaMemset(h->status_dev, 0, 2 * sizeof(unsigned int)) != cudaSuccess ||
+        cudaMalloc(&h->lut_arena_dev, (size_t)kLutSlots * 256 * sizeof(uint64_t)) != cudaSuccess) {
+        awe_destroy(h);
+        return AWE_ERR_CUDA;
+    }
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &h->encode_tiled, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess || !h->encode_tiled) {
+        awe_destroy(h);
+        return AWE_ERR_CUDA;
+    }
+    *out = h;
+    return AWE_OK;
+}
+
+extern "C" awe_status_t awe_destroy(awe_handle_t h) {
+    if (!h) return AWE_ERR_INVALID_ARG;
+    cudaSetDevice(h->device);
+    if (h->status_dev) cudaFree(h->status_dev);
+    if (h->lut_arena_dev) cudaFree(h->lut_arena_dev);
+    delete h;
+    return AWE_OK;
+}
+
+namespace awe {
+awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, cudaStream_t stream,
+                        const uint64_t** out) {
+    for (size_t i = 0; i < h->slots.size(); ++i) {
+        const auto& s = h->slots[i];
+        if (s.enc == enc && s.modulus == modulus && s.side == (int)side && s.dt == (int)dt) {
+            *out = h->lut_arena_dev + i * 256;
+            return AWE_OK;
+        }
+    }
+    if ((int)h->slots.size() >= kLutSlots) return AWE_ERR_UNSUPPORTED;
+    const SideTable* t;
+    if (!get_side_table(enc, modulus, side, dt, &t)) return AWE_ERR_UNSUPPORTED;
+    uint64_t* dst = h->lut_arena_dev + h->slots.size() * 256;
+    // The table lives in host memory owned by the library for the life of the process, so the
+    // copy may complete after this call returns.
+    if (cudaMemcpyAsync(dst, t->lut, 256 * sizeof(uint64_t), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return AWE_ERR_CUDA;
+    // Later calls may use another stream: make the table visible to all of them now.
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return AWE_ERR_CUDA;
+    h->slots.push_back({enc, modulus, (int)side, (int)dt});
+    *out = dst;
+    return AWE_OK;
+}
+}  // namespace awe
+
+static size_t out_elem_bytes(awe_out_dtype_t t) { return t == AWE_C_I64 ? 8 : (t == AWE_C_RES_I16 ? 2 : 4); }
+
+extern "C" size_t awe_host_staging_bytes(int enc, int modulus, int64_t M, int64_t N, int64_t K,
+                                         awe_out_dtype_t out_dt) {
+    if (!awe_workspace_bytes(enc, modulus, M, N, K)) return 0;
+    return (size_t)round_up(M * K, 256) + (size_t)round_up(K * N, 256) +
+           (size_t)round_up(M * N * (int64_t)out_elem_bytes(out_dt), 256);
+}
+
+extern "C" awe_status_t awe_gemm_exact(awe_handle_t h, const void* A_dev, awe_in_dtype_t a_dt, const void* B_dev,
+                                       awe_in_dtype_t b_dt, int64_t M, int64_t N, int64_t K, int enc, int modulus,
+                                       void* C_dev, awe_out_dtype_t out_dt, void* workspace_dev,
+                                       size_t workspace_bytes, void* stream) {
+    if (!h || !A_dev || !B_dev || !C_dev || !workspace_dev || M <= 0 || N <= 0 || K <= 0)
+        return AWE_ERR_INVALID_ARG;
+    const size_t need = awe_workspace_bytes(enc, modulus, M, N, K);
+    if (!need) return AWE_ERR_UNSUPPORTED;
+    if (workspace_bytes < need) return AWE_ERR_WORKSPACE;
+    if ((uintptr_t)workspace_dev % 256) return AWE_ERR_ALIGNMENT;
+    // Everything the later steps would reject is checked before the first launch.
+    if ((int)out_dt < 0 || (int)out_dt > 3) return AWE_ERR_INVALID_ARG;
+    awe_encoding_desc d;
+    awe_status_t s = awe_encoding_info(enc, modulus, &d);
+    if (s != AWE_OK) return s;
+    if ((d.modulus != 0) != (out_dt == AWE_C_RES_I16 || out_dt == AWE_C_RES_I32)) return AWE_ERR_UNSUPPORTED;
+    if ((uintptr_t)C_dev % out_elem_bytes(out_dt)) return AWE_ERR_ALIGNMENT;
+    const SideTable* t;
+    if (!get_side_table(enc, modulus, AWE_SIDE_A, a_dt, &t) || !get_side_table(enc, modulus, AWE_SIDE_B, b_dt, &t))
+        return AWE_ERR_UNSUPPORTED;
+    const int64_t amax = std::max(std::abs(d.a_lo), std::abs(d.a_hi));
+    const int64_t bmax = std::max(std::abs(d.b_lo), std::abs(d.b_hi));
+    if (out_dt == AWE_C_I32 && (__int128)amax * bmax * K >= ((__int128)1 << 31)) return AWE_ERR_RANGE;
+
+    uint8_t* pa = (uint8_t*)workspace_dev;
+    uint8_t* pb = pa + round_up((int64_t)awe_planes_bytes(enc, modulus, AWE_SIDE_A, M, K), 256);
+    if ((s = awe_encode(h, enc, modulus, AWE_SIDE_A, A_dev, a_dt, AWE_ROWMAJOR_RxK, M, K, K, pa, stream)) != AWE_OK)
+        return s;
+    if ((s = awe_encode(h, enc, modulus, AWE_SIDE_B, B_dev, b_dt, AWE_ROWMAJOR_KxR, N, K, N, pb, stream)) != AWE_OK)
+        return s;
+    return awe_gemm_planes(h, enc, modulus, pa, pb, M, N, K, C_dev, out_dt, N, 0, stream);
+}
+
+extern "C" awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, awe_in_dtype_t a_dt,
+                                            const void* B_host, awe_in_dtype_t b_dt, int64_t M, int64_t N, int64_t K,
+                                            int enc, int modulus, void* C_host, awe_out_dtype_t out_dt,
+                                            void* scratch_dev, size_t scratch_bytes, void* stream) {
+    if (!h || !A_host || !B_host || !C_host || !scratch_dev || M <= 0 || N <= 0 || K <= 0)
+        return AWE_ERR_INVALID_ARG;
+    if ((int)out_dt < 0 || (int)out_dt > 3) return AWE_ERR_INVALID_ARG;
+    const size_t ws = awe_workspace_bytes(enc, modulus, M, N, K);
+    const size_t staging = awe_host_staging_bytes(enc, modulus, M, N, K, out_dt);
+    if (!ws || !staging) return AWE_ERR_UNSUPPORTED;
+    if (scratch_bytes < ws + staging) return AWE_ERR_WORKSPACE;
+    if ((uintptr_t)scratch_dev % 256) return AWE_ERR_ALIGNMENT;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* base = (uint8_t*)scratch_dev;
+    uint8_t* dA = base + round_up((int64_t)ws, 256);
+    uint8_t* dB = dA + round_up(M * K, 256);
+    uint8_t* dC = dB + round_up(K * N, 256);
+    const size_t c_bytes = (size_t)M * N * out_elem_bytes(out_dt);
+    if (cudaMemcpyAsync(dA, A_host, (size_t)M * K, cudaMemcpyHostToDevice, st) != cudaSuccess) return AWE_ERR_CUDA;
+    if (cudaMemcpyAsync(dB, B_host, (size_t)K * N, cudaMemcpyHostToDevice, st) != cudaSuccess) return AWE_ERR_CUDA;
+    awe_status_t s = awe_gemm_exact(h, dA, a_dt, dB, b_dt, M, N, K, enc, modulus, dC, out_dt, base, ws, stream);
+    if (s != AWE_OK) return s;
+    if (cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return AWE_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return AWE_ERR_CUDA;
+    return AWE_OK;
+}
+
+extern "C" awe_status_t awe_last_device_status(awe_handle_t h, void* stream, int* site) {
+    if (!h) return AWE_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return AWE_ERR_CUDA;
+    unsigned int w[2] = {0, 0};
+    if (cudaMemcpy(w, h->status_dev, sizeof(w), cudaMemcpyDeviceToHost) != cudaSuccess) return AWE_ERR_CUDA;
+    if (w[0] != 0 && cudaMemset(h->status_dev, 0, sizeof(w)) != cudaSuccess) return AWE_ERR_CUDA;
+    if (site) *site = (int)w[1];
+    return (awe_status_t)w[0];
+}
+
+extern "C" int64_t awe_launch_count(awe_handle_t h) { return h ? h->launches : -1; }

@@ -1,0 +1,475 @@
+// FP4 products and fused integer reconstruction (Algorithm 1, third loop and last step).
+//
+// One persistent CTA per SM walks over 128 x 256 output tiles.  For every tile and every product
+// k it streams the K-major E2M1 planes alpha_k (A side) and beta_k (B side) through a TMA ->
+// shared-memory ring, multiplies them with tcgen05.mma kind::mxf4 (block scales held constant)
+// into an FP32 accumulator in tensor memory, and after every K segment (Section 3.4: short
+// enough that each partial sum is an integer below 2^24, hence exact) the epilogue warps drain
+// the accumulator, convert it to integers and add l_k times it to a register-resident 32-bit
+// running sum.  After the last product the sum is shifted by log2 D (Definition 4.1) or reduced
+// mod m (Section 5.3) and written once.
+//
+// 32-bit wrap-around is deliberate: sum_k l_k P_k is computed modulo 2^32, which equals the
+// true D*C whenever |D*C| < 2^31 (checked on the host), although single terms may exceed it.
+//
+// Warp roles: warp 0 lane 0 issues TMA loads, warp 1 lane 0 issues MMAs (warp 1 also owns the
+// tensor-memory allocation), warps 2..9 are the epilogue (warp w reads TMEM lanes 32*(w%4)..+31
+// and columns 128*((w-2)/4)..+127).  Every wait is bounded: when one expires the CTA records the
+// site in the status word, raises a shared abort flag and winds down normally.
+#include <cuda.h>
+
+#include <algorithm>
+
+#include "awe_internal.h"
+#include "ptx.cuh"
+
+namespace awe {
+namespace {
+
+constexpr int kTileM = 128;
+constexpr int kTileN = 256;
+constexpr int kBlockKBytes = 128;  // 256 E2M1 elements: one 128-byte swizzle row
+constexpr int kStages = 4;
+constexpr int kABytes = kTileM * kBlockKBytes;  // 16 KB
+constexpr int kBBytes = kTileN * kBlockKBytes;  // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kThreads = 320;
+constexpr int kEpiWarps = 8;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kAccCol = 0;
+constexpr uint32_t kSfaCol = 256;  // 16 columns of constant scale bytes each for A and B
+constexpr uint32_t kSfbCol = 272;
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+
+enum OutMode { OUT_I32 = 0, OUT_I64 = 1, OUT_RES_I16 = 2, OUT_RES_I32 = 3, OUT_RAW_F32 = 4 };
+
+struct GemmParams {
+    int M, N;
+    int tiles_m, tiles_n;
+    int kblock0;        // first 256-element K block of this launch
+    int num_kblocks;    // K blocks of this launch
+    int chunk_kblocks;  // K blocks per exact accumulation segment
+    int r;
+    int ia[AWE_MAX_PRODUCTS], ib[AWE_MAX_PRODUCTS], ell[AWE_MAX_PRODUCTS];
+    int log2D, modulus;
+    int out_mode, accumulate;
+    void* C;
+    long long ldc;
+    unsigned int* status;
+    int vec_store;     // C rows are 16-byte aligned: vector stores allowed
+    float acc_scale;   // accumulator value -> product of doubled integers
+    uint32_t sf_word;  // four copies of the UE8M0 scale byte
+};
+
+// mxf4 instruction descriptor: E2M1 x E2M1, both K-major, UE8M0 scales, M = 128, N = 256, dense K = 64.
+constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | (1u << 23) |
+                            ((uint32_t)(kTileM >> 4) << 24);
+
+struct Shared {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t tmem_full;
+    uint64_t tmem_empty;
+    uint32_t tmem_base;
+    volatile uint32_t abort_flag;
+};
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+
+__device__ __forceinline__ bool bounded_wait(Shared* sh, uint32_t bar, uint32_t parity, unsigned int* status,
+                                             int site) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = ptx::globaltimer_ns();
+    uint32_t polls = 0;
+    for (;;) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (sh->abort_flag) return false;
+        if ((++polls & 1023u) == 0 && ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
+            if (atomicCAS(status, 0u, (unsigned)AWE_ERR_TIMEOUT) == 0u) status[1] = (unsigned)site;
+            sh->abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int* tm, int* tn) {
+    constexpr int kGroupM = 8;
+    const int per_group = kGroupM * tiles_n;
+    const int group = t / per_group, in_group = t % per_group;
+    const int first_m = group * kGroupM;
+    const int gsize = min(tiles_m - first_m, kGroupM);
+    *tm = first_m + in_group % gsize;
+    *tn = in_group / gsize;
+}
+
+__device__ __forceinline__ int fast_mod(int x, int m, float inv_m) {
+    int q = __float2int_rz(__int2float_rn(x) * inv_m);
+    int r = x - q * m;
+    if (r < 0) r += m;
+    if (r >= m) r -= m;
+    if (r < 0) r += m;
+    return r;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const __grid_constant__ GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = ptx::smem_u32(smem_raw);
+    const uint32_t tiles_base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
+    Shared* sh = reinterpret_cast<Shared*>(smem_raw + (tiles_base - raw) + (size_t)kStages * kStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
+        }
+        ptx::mbar_init(ptx::smem_u32(&sh->tmem_full), 1);
+        ptx::mbar_init(ptx::smem_u32(&sh->tmem_empty), kEpiWarps);
+        sh->abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&map_a);
+        ptx::prefetch_tensormap(&map_b);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = sh->tmem_base;
+
+    // Constant block scales: every byte of 32 columns x 128 lanes holds the same UE8M0 value,
+    // so whatever bytes the MMA picks as scale factors, it reads that value.
+    if (warp >= 2 && warp < 6) {
+        const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
+        ptx::tmem_st_fill16(tmem + (lane_base << 16) + kSfaCol, p.sf_word);
+        ptx::tmem_st_fill16(tmem + (lane_base << 16) + kSfbCol, p.sf_word);
+        ptx::tmem_wait_st();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int chunks = (p.num_kblocks + p.chunk_kblocks - 1) / p.chunk_kblocks;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------------------------------------------------------- TMA producer
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                int tm, tn;
+                tile_coords(t, p.tiles_m, p.tiles_n, &tm, &tn);
+                for (int k = 0; k < p.r && ok; ++k) {
+                    for (int kb = 0; kb < p.num_kblocks; ++kb, ++it) {
+                        const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+                        if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->empty[s]), ph ^ 1u, p.status, 1))) break;
+                        const uint32_t bar = ptx::smem_u32(&sh->full[s]);
+                        ptx::mbar_arrive_expect_tx(bar, kStageBytes);
+                        const uint32_t a_dst = tiles_base + s * kStageBytes;
+                        const int x = (p.kblock0 + kb) * kBlockKBytes;
+                        ptx::tma_load_3d(a_dst, &map_a, bar, x, tm * kTileM, p.ia[k]);
+                        ptx::tma_load_3d(a_dst + kABytes, &map_b, bar, x, tn * kTileN, p.ib[k]);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------------------------------------------------------- MMA issuer
+            uint32_t it = 0, drains = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                for (int k = 0; k < p.r && ok; ++k) {
+                    for (int c = 0; c < chunks && ok; ++c, ++drains) {
+                        if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->tmem_empty), (drains & 1u) ^ 1u, p.status, 2)))
+                            break;
+                        ptx::tc_fence_after();
+                        const int kb_end = min(p.num_kblocks, (c + 1) * p.chunk_kblocks);
+                        for (int kb = c * p.chunk_kblocks; kb < kb_end; ++kb, ++it) {
+                            const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+                            if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->full[s]), ph, p.status, 3))) break;
+                            ptx::tc_fence_after();
+                            const uint32_t a_addr = tiles_base + s * kStageBytes;
+                            const uint64_t a_desc = ptx::smem_desc_k_sw128(a_addr);
+                            const uint64_t b_desc = ptx::smem_desc_k_sw128(a_addr + kABytes);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                // 64 elements = 32 bytes further along K inside the swizzle row
+                                ptx::mma_mxf4(tmem + kAccCol, a_desc + 2u * j, b_desc + 2u * j, kIdesc, tmem + kSfaCol,
+                                              tmem + kSfbCol, (kb > c * p.chunk_kblocks || j > 0) ? 1u : 0u);
+                            }
+                            ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));
+                        }
+                        if (ok) ptx::mma_commit(ptx::smem_u32(&sh->tmem_full));
+                    }
+                }
+            }
+        }
+    } else {
+        // -------------------------------------------------------------------- epilogue
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + kAccCol + (uint32_t)half * 128u;
+        const int m = p.modulus;
+        const float inv_m = m ? 1.0f / (float)m : 0.0f;
+        uint32_t drains = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            int tm, tn;
+            tile_coords(t, p.tiles_m, p.tiles_n, &tm, &tn);
+            uint32_t sum[128];
+#pragma unroll
+            for (int i = 0; i < 128; ++i) sum[i] = 0;
+            for (int k = 0; k < p.r && ok; ++k) {
+                const int ell = p.ell[k];
+                for (int c = 0; c < chunks && ok; ++c, ++drains) {
+                    ok = bounded_wait(sh, ptx::smem_u32(&sh->tmem_full), drains & 1u, p.status, 4);
+                    ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below need the whole warp
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        uint32_t v[32];
+                        ptx::tmem_ld_32x32(taddr + b * 32, v);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float f = __uint_as_float(v[i]) * p.acc_scale;
+                            if (p.out_mode == OUT_RAW_F32) {
+                                sum[b * 32 + i] = __float_as_uint(f);
+                            } else if (m) {
+                                const int pm = fast_mod(__float2int_rn(f), m, inv_m);
+                                sum[b * 32 + i] = (uint32_t)fast_mod((int)sum[b * 32 + i] + ell * pm, m, inv_m);
+                            } else {
+                                sum[b * 32 + i] += (uint32_t)ell * (uint32_t)__float2int_rn(f);
+                            }
+                        }
+                    }
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->tmem_empty));
+                }
+            }
+            if (!ok) break;
+            // ---- write the tile: this thread owns one row and 128 consecutive columns
+            const long long row = (long long)tm * kTileM + quarter * 32 + lane;
+            const int col0 = tn * kTileN + half * 128;
+            if (row < p.M) {
+                const int ncols = min(128, p.N - col0);
+                const int hi_res = (m + 1) / 2 - 1;
+                if (p.out_mode == OUT_I32 || p.out_mode == OUT_RES_I32 || p.out_mode == OUT_RAW_F32) {
+                    uint32_t* dst = reinterpret_cast<uint32_t*>(p.C) + row * p.ldc + col0;
+#pragma unroll
+                    for (int i = 0; i < 128; i += 4) {
+                        uint32_t o[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint32_t x = sum[i + j];
+                            if (p.out_mode == OUT_I32) x = (uint32_t)((int)x >> p.log2D);
+                            if (p.out_mode == OUT_RES_I32) x = (uint32_t)((int)x > hi_res ? (int)x - m : (int)x);
+                            o[j] = x;
+                        }
+                        if (p.vec_store && i + 4 <= ncols) {
+                            *reinterpret_cast<uint4*>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                if (i + j < ncols) dst[i + j] = o[j];
+                        }
+                    }
+                } else if (p.out_mode == OUT_I64) {
+                    long long* dst = reinterpret_cast<long long*>(p.C) + row * p.ldc + col0;
+#pragma unroll
+                    for (int i = 0; i < 128; i += 2) {
+                        long long o0 = (long long)((int)sum[i] >> p.log2D);
+                        long long o1 = (long long)((int)sum[i + 1] >> p.log2D);
+                        if (p.vec_store && i + 2 <= ncols) {
+                            if (p.accumulate) {
+                                const longlong2 old = *reinterpret_cast<longlong2*>(dst + i);
+                                o0 += old.x;
+                                o1 += old.y;
+                            }
+                            *reinterpret_cast<longlong2*>(dst + i) = make_longlong2(o0, o1);
+                        } else {
+                            if (i < ncols) dst[i] = p.accumulate ? dst[i] + o0 : o0;
+                            if (i + 1 < ncols) dst[i + 1] = p.accumulate ? dst[i + 1] + o1 : o1;
+                        }
+                    }
+                } else {  // OUT_RES_I16
+                    short* dst = reinterpret_cast<short*>(p.C) + row * p.ldc + col0;
+#pragma unroll
+                    for (int i = 0; i < 128; i += 8) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            int x0 = (int)sum[i + 2 * j], x1 = (int)sum[i + 2 * j + 1];
+                            x0 = x0 > hi_res ? x0 - m : x0;
+                            x1 = x1 > hi_res ? x1 - m : x1;
+                            w[j] = ((uint32_t)x0 & 0xFFFFu) | ((uint32_t)x1 << 16);
+                        }
+                        if (p.vec_store && i + 8 <= ncols) {
+                            *reinterpret_cast<uint4*>(dst + i) = make_uint4(w[0], w[1], w[2], w[3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                if (i + j < ncols) dst[i + j] = (short)((w[j >> 1] >> (16 * (j & 1))) & 0xFFFFu);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ------------------------------------------------------------------------ wind down
+    if (sh->abort_flag) {
+        // give copies and MMAs that are still in flight time to land before memory is released
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// planes: n_planes x rows x pitch bytes.  Box: 128 bytes of K x box_rows rows of one plane.
+awe_status_t make_plane_map(awe_ctx* h, const void* planes, int64_t rows, int64_t pitch, int n_planes,
+                            int box_rows, CUtensorMap* out) {
+    if (!h->encode_tiled) return AWE_ERR_CUDA;
+    cuuint64_t dims[3] = {(cuuint64_t)pitch, (cuuint64_t)rows, (cuuint64_t)n_planes};
+    cuuint64_t strides[2] = {(cuuint64_t)pitch, (cuuint64_t)pitch * (cuuint64_t)rows};
+    cuuint32_t box[3] = {(cuuint32_t)kBlockKBytes, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = ((EncodeTiledFn)h->encode_tiled)(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(planes),
+                                                  dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? AWE_OK : AWE_ERR_CUDA;
+}
+
+awe_status_t launch_gemm(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(awe_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) !=
+            cudaSuccess)
+            return AWE_ERR_CUDA;
+        attr_set = true;
+    }
+    p.tiles_m = (p.M + kTileM - 1) / kTileM;
+    p.tiles_n = (p.N + kTileN - 1) / kTileN;
+    p.status = h->status_dev;
+    const int grid = std::min(p.tiles_m * p.tiles_n, h->sm_count);
+    awe_gemm_kernel<<<grid, kThreads, kSmemBytes, st>>>(ma, mb, p);
+    if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
+    h->launches += 1;
+    return AWE_OK;
+}
+
+// UE8M0 scale 2^0 on both operands: the accumulator then holds (product of doubled integers)/4.
+constexpr uint32_t kScaleWord = 0x7F7F7F7Fu;
+constexpr float kAccScale = 4.0f;
+
+}  // namespace
+}  // namespace awe
+
+using namespace awe;
+
+extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, const void* planesA_dev,
+                                        const void* planesB_dev, int64_t M, int64_t N, int64_t K, void* C_dev,
+                                        awe_out_dtype_t out_dt, int64_t ldc, int64_t k_chunk, void* stream) {
+    if (!h || !planesA_dev || !planesB_dev || !C_dev || M <= 0 || N <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
+    if (M > (1 << 30) || N > (1 << 30) || K > (1ll << 36)) return AWE_ERR_INVALID_ARG;
+    if (ldc < N || k_chunk < 0 || (k_chunk % 256) != 0) return AWE_ERR_INVALID_ARG;
+    if ((int)out_dt < 0 || (int)out_dt > 3) return AWE_ERR_INVALID_ARG;
+    awe_encoding_desc d;
+    awe_status_t s = awe_encoding_info(enc, modulus, &d);
+    if (s != AWE_OK) return s;
+    const bool residue = d.modulus != 0;
+    if (residue != (out_dt == AWE_C_RES_I16 || out_dt == AWE_C_RES_I32)) return AWE_ERR_UNSUPPORTED;
+    const size_t elem = out_dt == AWE_C_I64 ? 8 : (out_dt == AWE_C_RES_I16 ? 2 : 4);
+    if ((uintptr_t)planesA_dev % 256 || (uintptr_t)planesB_dev % 256 || (uintptr_t)C_dev % elem)
+        return AWE_ERR_ALIGNMENT;
+    const int vec_store = ((uintptr_t)C_dev % 16 == 0) && (((size_t)ldc * elem) % 16 == 0);
+    // |C| <= max|a| max|b| K must fit the output type
+    const int64_t amax = std::max(std::abs(d.a_lo), std::abs(d.a_hi));
+    const int64_t bmax = std::max(std::abs(d.b_lo), std::abs(d.b_hi));
+    if (out_dt == AWE_C_I32 && (__int128)amax * bmax * K >= ((__int128)1 << 31)) return AWE_ERR_RANGE;
+
+    const int64_t pitch = plane_pitch_bytes(K);
+    CUtensorMap ma, mb;
+    if ((s = make_plane_map(h, planesA_dev, M, pitch, d.n_planes_a, kTileM, &ma)) != AWE_OK) return s;
+    if ((s = make_plane_map(h, planesB_dev, N, pitch, d.n_planes_b, kTileN, &mb)) != AWE_OK) return s;
+
+    GemmParams p = {};
+    p.M = (int)M;
+    p.N = (int)N;
+    p.r = d.r;
+    for (int k = 0; k < d.r; ++k) {
+        p.ia[k] = d.ia[k];
+        p.ib[k] = d.ib[k];
+        p.ell[k] = d.ell[k];
+    }
+    p.log2D = d.log2D;
+    p.modulus = d.modulus;
+    p.out_mode = (int)out_dt;
+    p.C = C_dev;
+    p.ldc = ldc;
+    p.vec_store = vec_store;
+    p.acc_scale = kAccScale;
+    p.sf_word = kScaleWord;
+    // exact accumulation segment (Section 3.4): a multiple of 256 not above K*
+    int64_t kc = k_chunk ? k_chunk : std::max<int64_t>(256, d.k_star / 256 * 256);
+    p.chunk_kblocks = (int)std::min<int64_t>(kc / 256, 1 << 20);
+    const int64_t total_kblocks = pitch / kBlockKBytes;
+    // 64-bit results: K is cut into launches whose own result fits 32 bits, added in int64
+    int64_t seg_kblocks = total_kblocks;
+    if (out_dt == AWE_C_I64 && !residue) {
+        int64_t seg = ((int64_t)1 << 30) / (amax * bmax * ((int64_t)1 << d.log2D));
+        seg_kblocks = std::max<int64_t>(1, std::min(total_kblocks, seg / 256));
+    }
+    if (residue) seg_kblocks = total_kblocks;
+    for (int64_t kb0 = 0; kb0 < total_kblocks; kb0 += seg_kblocks) {
+        p.kblock0 = (int)kb0;
+        p.num_kblocks = (int)std::min(seg_kblocks, total_kblocks - kb0);
+        p.accumulate = kb0 > 0;
+        if ((s = launch_gemm(h, ma, mb, p, (cudaStream_t)stream)) != AWE_OK) return s;
+    }
+    return AWE_OK;
+}
+
+extern "C" awe_status_t awe_fp4_product_raw(awe_handle_t h, const void* planeX_dev, const void* planeY_dev,
+                                            int64_t M, int64_t N, int64_t K, float* P_dev, int64_t ldp,
+                                            void* stream) {
+    if (!h || !planeX_dev || !planeY_dev || !P_dev || M <= 0 || N <= 0 || K <= 0 || ldp < N)
+        return AWE_ERR_INVALID_ARG;
+    if (M > (1 << 30) || N > (1 << 30) || K > (1ll << 30)) return AWE_ERR_INVALID_ARG;
+    if ((uintptr_t)planeX_dev % 256 || (uintptr_t)planeY_dev % 256 || (uintptr_t)P_dev % 4) return AWE_ERR_ALIGNMENT;
+    const int64_t pitch = plane_pitch_bytes(K);
+    CUtensorMap ma, mb;
+    awe_status_t s;
+    if ((s = make_plane_map(h, planeX_dev, M, pitch, 1, kTileM, &ma)) != AWE_OK) return s;
+    if ((s = make_plane_map(h, planeY_dev, N, pitch, 1, kTileN, &mb)) != AWE_OK) return s;
+    GemmParams p = {};
+    p.M = (int)M;
+    p.N = (int)N;
+    p.r = 1;
+    p.ell[0] = 1;
+    p.out_mode = OUT_RAW_F32;
+    p.C = P_dev;
+    p.ldc = ldp;
+    p.vec_store = ((uintptr_t)P_dev % 16 == 0) && ((ldp * 4) % 16 == 0);
+    p.acc_scale = kAccScale;
+    p.sf_word = kScaleWord;
+    p.num_kblocks = (int)(pitch / kBlockKBytes);
+    p.chunk_kblocks = p.num_kblocks;
+    return launch_gemm(h, ma, mb, p, (cudaStream_t)stream);
+}

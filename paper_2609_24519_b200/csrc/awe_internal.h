@@ -1,0 +1,67 @@
+// Internal declarations shared by the translation units of the AWE library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <mutex>
+#include <vector>
+
+#include "awe.h"
+
+namespace awe {
+
+constexpr int kMaxLimbs = 4;
+
+// One configuration record (Definition 4.1): weights, planes per product, integer
+// reconstruction coefficients, denominator 2^log2D, optional modulus (Section 5.3).
+struct Scheme {
+    int p = 0, q = 0, r = 0;
+    int w[kMaxLimbs] = {0}, v[kMaxLimbs] = {0};
+    int alpha[AWE_MAX_PRODUCTS][kMaxLimbs] = {{0}};
+    int beta[AWE_MAX_PRODUCTS][kMaxLimbs] = {{0}};
+    int ell[AWE_MAX_PRODUCTS] = {0};
+    int log2D = 0;
+    int modulus = 0;
+    int a_lo = -128, a_hi = 127, b_lo = -128, b_hi = 127;
+};
+
+// Stored planes of one side and the per-byte table derived from the record.
+struct SideTable {
+    int n_planes = 0;
+    int planes[AWE_MAX_PLANES][kMaxLimbs] = {{0}};
+    int index_of_product[AWE_MAX_PRODUCTS] = {0};
+    int c = 0;                         // largest |plane value| over the input range
+    int8_t value[256][AWE_MAX_PLANES]; // plane values for raw byte b (index b & 0xFF)
+    uint64_t lut[256];                 // E2M1 code of plane j in the low nibble of byte j
+};
+
+// Builds (and caches) scheme + tables; returns false if the encoding/modulus is not available.
+bool get_scheme(int enc, int modulus, Scheme* out);
+bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, const SideTable** out);
+awe_in_dtype_t natural_dtype(int enc, awe_side_t side);
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+inline int64_t plane_pitch_bytes(int64_t K) { return round_up(K, 256) / 2; }
+
+}  // namespace awe
+
+struct awe_ctx {
+    int device = 0;
+    int sm_count = 0;
+    unsigned int* status_dev = nullptr;  // [0] = status, [1] = site
+    uint64_t* lut_arena_dev = nullptr;   // kLutSlots tables of 256 x u64
+    struct LutSlot {
+        int enc, modulus, side, dt;
+    };
+    std::vector<LutSlot> slots;
+    int64_t launches = 0;
+    void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
+    std::mutex mu;
+};
+
+namespace awe {
+constexpr int kLutSlots = 96;
+// Device pointer of the 256-entry u64 table for (enc, modulus, side, dt); uploads on first use.
+awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_in_dtype_t dt,
+                        cudaStream_t stream, const uint64_t** out);
+}  // namespace awe

@@ -1,0 +1,193 @@
+"""FP4 products + fused reconstruction (Algorithm 1, third loop and last step; Section 3.4;
+Section 5.3) against the CPU oracle.  Integer results: the bar is bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import matmul as mm
+from oracle import pipeline as pl
+from oracle import rns
+from oracle import schemes as sc
+from paper_2609_24519_b200 import binding as b
+from paper_2609_24519_b200 import workloads as wl
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+INT8_ENCS = [(b.ENC_INT8_AWE6, "awe6"), (b.ENC_INT8_BASE13_9, "base13"), (b.ENC_INT8_AWE6_ALT, "alt")]
+
+
+# ------------------------------------------------------------------ raw FP4 product (Section 3.4)
+def _raw(X, Y):
+    got = gu.gpu_fp4_raw(X, Y, pl.pack_e2m1)
+    want = X.astype(np.int64) @ Y.astype(np.int64).T
+    assert np.array_equal(got, want.astype(np.float32)) and np.array_equal(got.astype(np.int64), want)
+
+
+def test_raw_product_random_planes():
+    rng = np.random.default_rng(2)
+    S = np.array(sc.S, dtype=np.int8)
+    for (M, N, K) in [(128, 256, 256), (100, 200, 300), (384, 512, 4096), (1, 1, 64), (129, 257, 257)]:
+        _raw(rng.choice(S, (M, K)), rng.choice(S, (N, K)))
+
+
+def test_raw_product_single_nonzero_and_position():
+    X = np.zeros((128, 512), dtype=np.int8)
+    Y = np.zeros((256, 512), dtype=np.int8)
+    X[77, 301] = -6
+    Y[200, 301] = 12
+    Y[13, 300] = 8
+    _raw(X, Y)
+
+
+def test_accumulation_is_exact_up_to_2_24():
+    """Section 3.4: planes of +-12 at K = 116,480 give |P| = 144 K = 16,773,120 < 2^24."""
+    K = 116480
+    assert 144 * K < 2 ** 24 and K <= sc.k_star(12, 12)
+    X = np.full((128, K), 12, dtype=np.int8)
+    Y = np.full((256, K), 12, dtype=np.int8)
+    Y[1::2] = -12
+    _raw(X, Y)
+
+
+def test_small_terms_survive_next_to_a_large_partial_sum():
+    """Adversarial order: the sum first climbs close to 2^24, then only tiny products of
+    both signs follow.  Any alignment that dropped low bits would lose them."""
+    rng = np.random.default_rng(3)
+    K1, K2 = 116000, 448
+    X = np.full((128, K1 + K2), 12, dtype=np.int8)
+    Y = np.full((256, K1 + K2), 12, dtype=np.int8)
+    X[:, K1:] = rng.choice(np.array([-1, 1, 2, -3], dtype=np.int8), (128, K2))
+    Y[:, K1:] = rng.choice(np.array([-1, 1, 3, -2], dtype=np.int8), (256, K2))
+    X[64:, :K1] = -12                                   # half the rows climb towards -2^24
+    assert 144 * K1 + 9 * K2 < 2 ** 24
+    _raw(X, Y)
+    # and the reverse order: small terms first, large ones after
+    _raw(np.ascontiguousarray(X[:, ::-1]), np.ascontiguousarray(Y[:, ::-1]))
+
+
+# ------------------------------------------------------------------ whole procedure
+@pytest.mark.parametrize("enc,name", INT8_ENCS)
+def test_config1_bit_exact(enc, name):
+    A, B = wl.make_inputs(wl.config1())
+    assert np.array_equal(gu.gpu_gemm_exact(A, B, enc, b.C_I32), mm.matmul_i64(A, B))
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1), (130, 270, 300), (257, 513, 1030), (640, 768, 2304), (127, 255, 257)])
+@pytest.mark.parametrize("enc,name", INT8_ENCS)
+def test_ragged_shapes_int8(enc, name, shape):
+    M, N, K = shape
+    A, B = wl.make_inputs(wl.small("t", M, N, K, seed=M + N + K))
+    want = mm.matmul_i64(A, B)
+    assert np.array_equal(gu.gpu_gemm_exact(A, B, enc, b.C_I32), want)
+    assert np.array_equal(gu.gpu_gemm_exact(A, B, enc, b.C_I64), want)
+
+
+def test_closed_forms_on_gpu():
+    K = 777
+    A = np.full((130, K), -128, dtype=np.int8)
+    B = np.full((K, 260), -128, dtype=np.int8)
+    assert np.all(gu.gpu_gemm_exact(A, B, b.ENC_INT8_AWE6, b.C_I32) == 16384 * K)
+    Bm = np.random.default_rng(3).integers(-128, 128, (200, 300), dtype=np.int8)
+    C = gu.gpu_gemm_exact(np.eye(200, dtype=np.int8), Bm, b.ENC_INT8_AWE6, b.C_I32)
+    assert np.array_equal(C, Bm.astype(np.int32))
+
+
+def test_int4_x_int8():
+    for (M, N, K) in [(256, 512, 512), (130, 270, 300)]:
+        A, B = wl.make_inputs(wl.small("t", M, N, K, "int4", "int8", seed=9))
+        got = gu.gpu_gemm_exact(A, B, b.ENC_INT4xINT8_AWE4, b.C_I32, a_dt=b.I4_IN_I8)
+        assert np.array_equal(got, mm.matmul_i64(A, B))
+
+
+@pytest.mark.parametrize("m", rns.RNS_SET_FP64)
+def test_residue_form_every_modulus_of_the_set(m):
+    A, B = wl.make_inputs(wl.small("t", 192, 320, 1100, "residue", "residue", seed=m, modulus=m))
+    want = mm.mod_symmetric(mm.matmul_i64(A, B), m)
+    assert np.array_equal(gu.gpu_gemm_exact(A, B, b.ENC_MOD_M, b.C_RES_I16, modulus=m), want)
+    assert np.array_equal(gu.gpu_gemm_exact(A, B, b.ENC_MOD_M, b.C_RES_I32, modulus=m), want)
+
+
+def test_residue_form_accepts_any_int8_input():
+    A, B = wl.make_inputs(wl.small("t", 128, 256, 512, seed=4))
+    want = mm.mod_symmetric(mm.matmul_i64(A, B), 61)
+    assert np.array_equal(gu.gpu_gemm_exact(A, B, b.ENC_MOD_M, b.C_RES_I16, modulus=61), want)
+
+
+@pytest.mark.parametrize("k_chunk", [0, 256, 512, 2048])
+def test_forced_k_segments_worst_case_inputs(k_chunk):
+    """Section 3.4 / 6.1: segmenting K and adding the segments in integers changes nothing."""
+    w = wl.small("t", 256, 512, 4096, "extreme", "extreme", seed=4)
+    A, B = wl.make_inputs(w)
+    want = mm.matmul_i64(A, B)
+    pa = gu.gpu_encode(b.ENC_INT8_AWE6, 0, b.SIDE_A, A)
+    pb = gu.gpu_encode(b.ENC_INT8_AWE6, 0, b.SIDE_B, np.ascontiguousarray(B.T))
+    for out in (b.C_I32, b.C_I64):
+        got = gu.gpu_gemm_planes(pa, pb, w.M, w.N, w.K, b.ENC_INT8_AWE6, out, k_chunk=k_chunk)
+        assert np.array_equal(got, want)
+
+
+def test_int64_output_beyond_32_bits():
+    """K = 2^18 with all entries -128: C = 2^14 K = 2^32, needs the 64-bit path."""
+    M, N, K = 128, 256, 1 << 18
+    A = np.full((M, K), -128, dtype=np.int8)
+    B = np.full((K, N), -128, dtype=np.int8)
+    B[:, 1::2] = 127
+    got = gu.gpu_gemm_exact(A, B, b.ENC_INT8_AWE6, b.C_I64)
+    assert np.all(got[:, 0::2] == (1 << 32)) and np.all(got[:, 1::2] == -128 * 127 * K)
+    with pytest.raises(b.AweError) as e:
+        gu.gpu_gemm_exact(A, B, b.ENC_INT8_AWE6, b.C_I32)
+    assert e.value.status == 5
+
+
+def test_planes_entry_with_leading_dimension_and_guard_columns():
+    w = wl.small("t", 130, 200, 300, seed=12)
+    A, B = wl.make_inputs(w)
+    pa = gu.gpu_encode(b.ENC_INT8_AWE6, 0, b.SIDE_A, A)
+    pb = gu.gpu_encode(b.ENC_INT8_AWE6, 0, b.SIDE_B, np.ascontiguousarray(B.T))
+    for ldc in (200, 203, 208):
+        got = gu.gpu_gemm_planes(pa, pb, w.M, w.N, w.K, b.ENC_INT8_AWE6, b.C_I32, ldc=ldc)
+        assert np.array_equal(got[:, :200], mm.matmul_i64(A, B))
+        assert np.all(got[:, 200:] == 77)                  # nothing written past N
+
+
+def test_results_are_reproducible_run_to_run():
+    A, B = wl.make_inputs(wl.small("t", 512, 768, 2048, seed=31))
+    first = gu.gpu_gemm_exact(A, B, b.ENC_INT8_AWE6, b.C_I32)
+    for _ in range(10):
+        assert np.array_equal(gu.gpu_gemm_exact(A, B, b.ENC_INT8_AWE6, b.C_I32), first)
+
+
+def test_host_buffer_entry_point():
+    h = gu.handle()
+    w = wl.small("t", 300, 520, 1000, seed=17)
+    A, B = wl.make_inputs(w)
+    Ah, Bh = torch.from_numpy(A).pin_memory(), torch.from_numpy(B).pin_memory()
+    Ch = torch.zeros((w.M, w.N), dtype=torch.int32).pin_memory()
+    nbytes = b.awe_workspace_bytes(b.ENC_INT8_AWE6, 0, w.M, w.N, w.K) + \
+        b.awe_host_staging_bytes(b.ENC_INT8_AWE6, 0, w.M, w.N, w.K, b.C_I32)
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    b.awe_gemm_exact_host(h, Ah, b.I8, Bh, b.I8, w.M, w.N, w.K, b.ENC_INT8_AWE6, 0, Ch, b.C_I32, scratch)
+    assert np.array_equal(Ch.numpy(), mm.matmul_i64(A, B))
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    h = gu.handle()
+    n0 = b.awe_launch_count(h)
+    A = torch.zeros((256, 256), dtype=torch.int8, device="cuda")
+    C = torch.zeros((256, 256), dtype=torch.int32, device="cuda")
+    ws = torch.empty(b.awe_workspace_bytes(b.ENC_INT8_AWE6, 0, 256, 256, 256) + 256, dtype=torch.uint8, device="cuda")
+    def call(**kw):
+        args = dict(A=A, a_dt=b.I8, B=A, b_dt=b.I8, M=256, N=256, K=256, enc=b.ENC_INT8_AWE6, modulus=0, C=C,
+                    out_dt=b.C_I32, workspace=ws)
+        args.update(kw)
+        b.awe_gemm_exact(h, **args)
+    for kw, status in [(dict(M=0), 1), (dict(enc=99), 2), (dict(modulus=7), 2), (dict(out_dt=b.C_RES_I16), 2),
+                       (dict(workspace=ws[:1024]), 3), (dict(workspace=ws[1:]), 4), (dict(A=None), 1),
+                       (dict(enc=b.ENC_INT4xINT8_AWE4), 2)]:     # int8 data on the int4 side
+        with pytest.raises(b.AweError) as e:
+            call(**kw)
+        assert e.value.status == status, kw
+    with pytest.raises(b.AweError):
+        b.awe_encoding_info(b.ENC_MOD_M, 170)
+    assert b.awe_launch_count(h) == n0

@@ -1,0 +1,70 @@
+"""The C-ABI library loads, exports every symbol include/awe.h declares, and its host-side
+tables agree with the oracle's independently built ones (no GPU, no compute calls)."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import pipeline as pl
+from oracle import rns
+from oracle import schemes as sc
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2609_24519_b200 import build
+    build.build()
+    from paper_2609_24519_b200 import binding
+    return binding
+
+
+def test_every_declared_symbol_is_exported(b):
+    header = open(os.path.join(ROOT, "include", "awe.h")).read()
+    declared = set(re.findall(r"\b(awe_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(b.EXPORTS)
+    L = b.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_records_match_the_paper_and_the_oracle(b):
+    for enc, s in ((b.ENC_INT8_AWE6, sc.AWE6), (b.ENC_INT8_AWE6_ALT, sc.AWE6_ALT),
+                   (b.ENC_INT8_BASE13_9, sc.BASE13_9), (b.ENC_INT4xINT8_AWE4, sc.AWE4)):
+        d = b.awe_encoding_info(enc)
+        assert d.r == s.r and list(d.ell)[:d.r] == list(s.ell) and d.log2D == s.log2D
+        assert list(d.ia)[:d.r] == s.plane_index("A") and list(d.ib)[:d.r] == s.plane_index("B")
+        assert d.n_planes_a == len(s.stored_planes("A")) and d.n_planes_b == len(s.stored_planes("B"))
+    d = b.awe_encoding_info(b.ENC_INT8_AWE6)
+    assert (d.c_a, d.c_b, d.k_star) == (6, 6, 466033)
+    d = b.awe_encoding_info(b.ENC_INT4xINT8_AWE4)
+    assert (d.c_a, d.c_b, d.k_star) == (3, 8, 699050)
+
+
+def test_tables_match_the_oracle_tables(b):
+    idx = np.arange(-128, 128) & 0xFF
+    for enc, s in ((b.ENC_INT8_AWE6, sc.AWE6), (b.ENC_INT8_AWE6_ALT, sc.AWE6_ALT), (b.ENC_INT8_BASE13_9, sc.BASE13_9)):
+        for side, name in ((b.SIDE_A, "A"), (b.SIDE_B, "B")):
+            assert np.array_equal(b.awe_encoding_lut(enc, 0, side)[idx], pl.plane_lut(s, name, -128, 127))
+    lut = b.awe_encoding_lut(b.ENC_INT4xINT8_AWE4, 0, b.SIDE_A, b.I4_IN_I8)
+    assert np.array_equal(lut[np.arange(-8, 8) & 0xFF], pl.plane_lut(sc.AWE4, "A", -8, 7))
+    assert np.array_equal(b.awe_encoding_lut(b.ENC_INT4xINT8_AWE4, 0, b.SIDE_B)[idx],
+                          pl.plane_lut(sc.AWE4, "B", -128, 127))
+    for m in rns.RNS_SET_FP64 + (2, 10, 37, 91, 100, 169):
+        s = sc.mod_scheme(m)
+        d = b.awe_encoding_info(b.ENC_MOD_M, m)
+        assert d.r == s.r and list(d.ell)[:d.r] == list(s.ell) and d.modulus == m
+        assert np.array_equal(b.awe_encoding_lut(b.ENC_MOD_M, m, b.SIDE_A)[idx], pl.plane_lut(s, "A", -128, 127))
+
+
+def test_sizes_and_host_side_rejections(b):
+    assert b.awe_planes_bytes(b.ENC_INT8_AWE6, 0, b.SIDE_A, 100, 300) == 6 * 100 * 256
+    assert b.awe_planes_bytes(b.ENC_INT8_BASE13_9, 0, b.SIDE_B, 8192, 8192) == 3 * 8192 * 4096
+    assert b.awe_workspace_bytes(b.ENC_INT8_AWE6, 0, 8192, 8192, 8192) == 2 * 6 * 8192 * 4096
+    assert b.awe_planes_bytes(99, 0, b.SIDE_A, 10, 10) == 0
+    assert b.awe_workspace_bytes(b.ENC_MOD_M, 170, 10, 10, 10) == 0
+    with pytest.raises(b.AweError):
+        b.awe_encoding_info(b.ENC_INT8_AWE6, 7)
+    assert "workspace" in b.status_string(3)
