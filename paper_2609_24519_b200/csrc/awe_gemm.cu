@@ -1,7 +1,12 @@
 // FP4 products and fused integer reconstruction (Algorithm 1, third loop and last step).
 //
-// One persistent CTA per SM walks over 128 x 256 output tiles.  For every tile and every product
-// k it streams the K-major E2M1 planes alpha_k (A side) and beta_k (B side) through a TMA ->
+// One persistent CTA per SM.  In the default variant two CTAs on neighbouring SMs form a pair
+// (a cluster of two) that shares one 256 x 256 output tile: each CTA loads its own 128 rows of
+// the A plane and its own 128 of the 256 rows of the B plane, CTA 0 issues one MMA for both
+// (cta_group::2: the halves of B are exchanged by the hardware, which halves the shared-memory
+// traffic per flop), and each CTA keeps and drains the 128 x 256 accumulator of its own rows.
+// The single-CTA variant works on 128 x 256 tiles alone.  For every tile and every product
+// k a CTA streams the K-major E2M1 planes alpha_k (A side) and beta_k (B side) through a TMA ->
 // shared-memory ring, multiplies them with tcgen05.mma kind::mxf4 (block scales held constant)
 // into an FP32 accumulator in tensor memory, and after every K segment (Section 3.4: short
 // enough that each partial sum is an integer below 2^24, hence exact) the epilogue warps drain
@@ -19,6 +24,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "awe_internal.h"
 #include "ptx.cuh"
@@ -26,20 +32,31 @@
 namespace awe {
 namespace {
 
-constexpr int kTileM = 128;
+constexpr int kTileM = 128;  // rows of A (and of the accumulator) per CTA
 constexpr int kTileN = 256;
 constexpr int kBlockKBytes = 128;  // 256 E2M1 elements: one 128-byte swizzle row
-constexpr int kStages = 4;
 constexpr int kABytes = kTileM * kBlockKBytes;  // 16 KB
-constexpr int kBBytes = kTileN * kBlockKBytes;  // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;
+
+// Per-variant sizes: a CTA of a pair stages only half of the B tile.
+template <bool kPair>
+struct Cfg {
+    static constexpr int kBRows = kPair ? kTileN / 2 : kTileN;
+    static constexpr int kBBytes = kBRows * kBlockKBytes;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kStages = kPair ? 6 : 4;
+    static constexpr int kCtas = kPair ? 2 : 1;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+    // mxf4 instruction descriptor: E2M1 x E2M1, both K-major, UE8M0 scales, dense K = 64
+    static constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | (1u << 23) |
+                                       ((uint32_t)((kTileM * kCtas) >> 4) << 24);
+};
+constexpr int kMaxStages = 6;
 constexpr int kThreads = 320;
 constexpr int kEpiWarps = 8;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAccCol = 0;
 constexpr uint32_t kSfaCol = 256;  // 16 columns of constant scale bytes each for A and B
 constexpr uint32_t kSfbCol = 272;
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
 
 enum OutMode { OUT_I32 = 0, OUT_I64 = 1, OUT_RES_I16 = 2, OUT_RES_I32 = 3, OUT_RAW_F32 = 4 };
 
@@ -61,13 +78,9 @@ struct GemmParams {
     uint32_t sf_word;  // four copies of the UE8M0 scale byte
 };
 
-// mxf4 instruction descriptor: E2M1 x E2M1, both K-major, UE8M0 scales, M = 128, N = 256, dense K = 64.
-constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | (1u << 23) |
-                            ((uint32_t)(kTileM >> 4) << 24);
-
 struct Shared {
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
     uint64_t tmem_full;
     uint64_t tmem_empty;
     uint32_t tmem_base;
@@ -111,9 +124,18 @@ __device__ __forceinline__ int fast_mod(int x, int m, float inv_m) {
     return r;
 }
 
+template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ GemmParams p) {
+    using C = Cfg<kPair>;
+    constexpr int kStages = C::kStages;
+    constexpr int kStageBytes = C::kStageBytes;
+    constexpr uint32_t kIdesc = C::kIdesc;
+    // rank of this CTA inside its pair; workers are pairs (or single CTAs)
+    const uint32_t rank = kPair ? ptx::cluster_ctarank() : 0u;
+    const int worker = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int num_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
@@ -126,18 +148,24 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
         }
         ptx::mbar_init(ptx::smem_u32(&sh->tmem_full), 1);
-        ptx::mbar_init(ptx::smem_u32(&sh->tmem_empty), kEpiWarps);
+        ptx::mbar_init(ptx::smem_u32(&sh->tmem_empty), kEpiWarps * C::kCtas);
         sh->abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&map_a);
         ptx::prefetch_tensormap(&map_b);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), kTmemCols);
-        ptx::tmem_relinquish();
+        if (kPair) {
+            ptx::tmem_alloc_pair(ptx::smem_u32(&sh->tmem_base), kTmemCols);
+            ptx::tmem_relinquish_pair();
+        } else {
+            ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), kTmemCols);
+            ptx::tmem_relinquish();
+        }
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (kPair) ptx::cluster_sync_all();  // the other CTA's barriers are initialised before anyone signals them
     ptx::tc_fence_after();
     const uint32_t tmem = sh->tmem_base;
 
@@ -161,29 +189,39 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // ---------------------------------------------------------------- TMA producer
             uint32_t it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            for (int t = worker; t < num_tiles && ok; t += num_workers) {
                 int tm, tn;
                 tile_coords(t, p.tiles_m, p.tiles_n, &tm, &tn);
+                const int row_a = (tm * C::kCtas + (int)rank) * kTileM;
+                const int row_b = tn * kTileN + (int)rank * C::kBRows;
                 for (int k = 0; k < p.r && ok; ++k) {
                     for (int kb = 0; kb < p.num_kblocks; ++kb, ++it) {
                         const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
                         if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->empty[s]), ph ^ 1u, p.status, 1))) break;
                         const uint32_t bar = ptx::smem_u32(&sh->full[s]);
-                        ptx::mbar_arrive_expect_tx(bar, kStageBytes);
                         const uint32_t a_dst = tiles_base + s * kStageBytes;
                         const int x = (p.kblock0 + kb) * kBlockKBytes;
-                        ptx::tma_load_3d(a_dst, &map_a, bar, x, tm * kTileM, p.ia[k]);
-                        ptx::tma_load_3d(a_dst + kABytes, &map_b, bar, x, tn * kTileN, p.ib[k]);
+                        if (kPair) {
+                            // both CTAs report their bytes to CTA 0's barrier, which expects the sum
+                            if (rank == 0) ptx::mbar_arrive_expect_tx(bar, 2 * kStageBytes);
+                            const uint32_t bar0 = ptx::map_to_cta(bar, 0);
+                            ptx::tma_load_3d_pair(a_dst, &map_a, bar0, x, row_a, p.ia[k]);
+                            ptx::tma_load_3d_pair(a_dst + kABytes, &map_b, bar0, x, row_b, p.ib[k]);
+                        } else {
+                            ptx::mbar_arrive_expect_tx(bar, kStageBytes);
+                            ptx::tma_load_3d(a_dst, &map_a, bar, x, row_a, p.ia[k]);
+                            ptx::tma_load_3d(a_dst + kABytes, &map_b, bar, x, row_b, p.ib[k]);
+                        }
                     }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             // ---------------------------------------------------------------- MMA issuer
             uint32_t it = 0, drains = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            for (int t = worker; t < num_tiles && ok; t += num_workers) {
                 for (int k = 0; k < p.r && ok; ++k) {
                     for (int c = 0; c < chunks && ok; ++c, ++drains) {
                         if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->tmem_empty), (drains & 1u) ^ 1u, p.status, 2)))
@@ -200,12 +238,22 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 // 64 elements = 32 bytes further along K inside the swizzle row
-                                ptx::mma_mxf4(tmem + kAccCol, a_desc + 2u * j, b_desc + 2u * j, kIdesc, tmem + kSfaCol,
-                                              tmem + kSfbCol, (kb > c * p.chunk_kblocks || j > 0) ? 1u : 0u);
+                                const uint32_t acc = (kb > c * p.chunk_kblocks || j > 0) ? 1u : 0u;
+                                if (kPair)
+                                    ptx::mma_mxf4_pair(tmem + kAccCol, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
+                                                       tmem + kSfaCol, tmem + kSfbCol, acc);
+                                else
+                                    ptx::mma_mxf4(tmem + kAccCol, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
+                                                  tmem + kSfaCol, tmem + kSfbCol, acc);
                             }
-                            ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));
+                            // frees the stage in both CTAs of a pair
+                            if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->empty[s]), 3);
+                            else ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));
                         }
-                        if (ok) ptx::mma_commit(ptx::smem_u32(&sh->tmem_full));
+                        if (ok) {
+                            if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->tmem_full), 3);
+                            else ptx::mma_commit(ptx::smem_u32(&sh->tmem_full));
+                        }
                     }
                 }
             }
@@ -218,7 +266,9 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const float inv_m = m ? 1.0f / (float)m : 0.0f;
         uint32_t drains = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        const uint32_t tmem_empty_bar = kPair ? ptx::map_to_cta(ptx::smem_u32(&sh->tmem_empty), 0)
+                                              : ptx::smem_u32(&sh->tmem_empty);
+        for (int t = worker; t < num_tiles && ok; t += num_workers) {
             int tm, tn;
             tile_coords(t, p.tiles_m, p.tiles_n, &tm, &tn);
             uint32_t sum[128];
@@ -251,12 +301,15 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     }
                     ptx::tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->tmem_empty));
+                    if (lane == 0) {
+                        if (kPair) ptx::mbar_arrive_cluster(tmem_empty_bar);
+                        else ptx::mbar_arrive(tmem_empty_bar);
+                    }
                 }
             }
             if (!ok) break;
             // ---- write the tile: this thread owns one row and 128 consecutive columns
-            const long long row = (long long)tm * kTileM + quarter * 32 + lane;
+            const long long row = (long long)(tm * C::kCtas + (int)rank) * kTileM + quarter * 32 + lane;
             const int col0 = tn * kTileN + half * 128;
             if (row < p.M) {
                 const int ncols = min(128, p.N - col0);
@@ -331,9 +384,11 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (kPair) ptx::cluster_sync_all();  // neither CTA leaves while the other may still signal it
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem, kTmemCols);
+        if (kPair) ptx::tmem_dealloc_pair(tmem, kTmemCols);
+        else ptx::tmem_dealloc(tmem, kTmemCols);
     }
 }
 
@@ -356,23 +411,52 @@ awe_status_t make_plane_map(awe_ctx* h, const void* planes, int64_t rows, int64_
     return r == CUDA_SUCCESS ? AWE_OK : AWE_ERR_CUDA;
 }
 
-awe_status_t launch_gemm(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
+// The pair variant is the default; AWE_GEMM_SINGLE_CTA=1 in the environment selects the other.
+bool use_pairs() {
+    static const bool v = [] {
+        const char* e = getenv("AWE_GEMM_SINGLE_CTA");
+        return !(e && e[0] == '1');
+    }();
+    return v;
+}
+
+template <bool kPair>
+awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p,
+                            cudaStream_t st) {
+    using C = Cfg<kPair>;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(awe_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(awe_gemm_kernel<kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)C::kSmemBytes) != cudaSuccess)
             return AWE_ERR_CUDA;
         attr_set = true;
     }
-    p.tiles_m = (p.M + kTileM - 1) / kTileM;
+    p.tiles_m = (p.M + kTileM * C::kCtas - 1) / (kTileM * C::kCtas);
     p.tiles_n = (p.N + kTileN - 1) / kTileN;
     p.status = h->status_dev;
-    const int grid = std::min(p.tiles_m * p.tiles_n, h->sm_count);
-    awe_gemm_kernel<<<grid, kThreads, kSmemBytes, st>>>(ma, mb, p);
-    if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
+    const int workers = std::min(p.tiles_m * p.tiles_n, h->sm_count / C::kCtas);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(workers * C::kCtas));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C::kCtas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair>, ma, mb, p) != cudaSuccess) return AWE_ERR_CUDA;
     h->launches += 1;
     return AWE_OK;
 }
+
+awe_status_t launch_gemm(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
+    return use_pairs() ? launch_variant<true>(h, ma, mb, p, st) : launch_variant<false>(h, ma, mb, p, st);
+}
+
+int b_box_rows() { return use_pairs() ? Cfg<true>::kBRows : Cfg<false>::kBRows; }
 
 // UE8M0 scale 2^0 on both operands: the accumulator then holds (product of doubled integers)/4.
 constexpr uint32_t kScaleWord = 0x7F7F7F7Fu;
@@ -407,7 +491,7 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
     const int64_t pitch = plane_pitch_bytes(K);
     CUtensorMap ma, mb;
     if ((s = make_plane_map(h, planesA_dev, M, pitch, d.n_planes_a, kTileM, &ma)) != AWE_OK) return s;
-    if ((s = make_plane_map(h, planesB_dev, N, pitch, d.n_planes_b, kTileN, &mb)) != AWE_OK) return s;
+    if ((s = make_plane_map(h, planesB_dev, N, pitch, d.n_planes_b, b_box_rows(), &mb)) != AWE_OK) return s;
 
     GemmParams p = {};
     p.M = (int)M;
@@ -457,7 +541,7 @@ extern "C" awe_status_t awe_fp4_product_raw(awe_handle_t h, const void* planeX_d
     CUtensorMap ma, mb;
     awe_status_t s;
     if ((s = make_plane_map(h, planeX_dev, M, pitch, 1, kTileM, &ma)) != AWE_OK) return s;
-    if ((s = make_plane_map(h, planeY_dev, N, pitch, 1, kTileN, &mb)) != AWE_OK) return s;
+    if ((s = make_plane_map(h, planeY_dev, N, pitch, 1, b_box_rows(), &mb)) != AWE_OK) return s;
     GemmParams p = {};
     p.M = (int)M;
     p.N = (int)N;
