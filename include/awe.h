@@ -160,6 +160,36 @@ awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, awe_in_dtyp
                                  void* C_host, awe_out_dtype_t out_dt, void* scratch_dev, size_t scratch_bytes,
                                  void* stream);
 
+/* Largest awe_workspace_bytes() a problem may need to go through awe_gemm_exact_static: 24 MiB,
+ * e.g. INT8xINT8 with the 6-product encoding up to M = N = K = 2048. */
+#define AWE_STATIC_WORKSPACE_BYTES (24u << 20)
+
+/* The same product as awe_gemm_exact for callers that must not allocate device memory and so
+ * cannot own a handle (awe_create calls cudaMalloc) or a workspace: code running inside a
+ * runtime's execute hook that forbids allocation, in a process whose memory pool already holds
+ * all of the GPU's memory so that cudaMalloc would fail, or on a latency-critical path that cannot
+ * take cudaMalloc's device-wide synchronisation.  (The paper has no counterpart; it is a
+ * deployment convenience.)  All device scratch -- planes, encode tables, status word -- comes from
+ * one array built into the library image: AWE_STATIC_WORKSPACE_BYTES + ~200 KB, resident on every
+ * GPU that loads the library until the process exits.  The call uses the CURRENT device, makes no
+ * cudaMalloc / cudaFree, and enqueues the same kernels as awe_gemm_exact on `stream`.
+ *   - A_dev, B_dev, C_dev, dtypes, sizes, enc, modulus, out_dt: exactly as for awe_gemm_exact
+ *     (A: M x K, B: K x N, C: M x N, all row-major and dense).
+ *   - AWE_ERR_WORKSPACE if awe_workspace_bytes(enc, modulus, M, N, K) exceeds
+ *     AWE_STATIC_WORKSPACE_BYTES; nothing is enqueued then.
+ *   - The first call on a device looks up the array's device address and the device's properties
+ *     and clears the status word; the first use of an encoding on a device uploads its tables and
+ *     waits for that copy.  Make those first calls before any stream capture.
+ *   - Every call on a device shares the one array, which keeps the previous call's planes: calls
+ *     whose kernels could overlap on the GPU (different streams, or several host threads) race
+ *     and must be serialised by the caller.  Nothing in it needs to start at zero except the status
+ *     word, which the library clears itself.
+ *   - A bounded device-side wait that expired during an earlier call is returned (as
+ *     AWE_ERR_TIMEOUT, once) by the first later call that finds `stream` idle. */
+awe_status_t awe_gemm_exact_static(const void* A_dev, awe_in_dtype_t a_dt, const void* B_dev, awe_in_dtype_t b_dt,
+                                   int64_t M, int64_t N, int64_t K, int enc, int modulus, void* C_dev,
+                                   awe_out_dtype_t out_dt, void* stream);
+
 /* One raw FP4 product P = X.Y^T with FP32 accumulation over all of K in a single segment
  * (Algorithm 1's "FP4-GEMM" alone; Section 3.4 is the claim this lets a test probe).
  * planeX_dev: M x pitch bytes, planeY_dev: N x pitch bytes, pitch = round_up(K,256)/2, packed E2M1;

@@ -24,10 +24,11 @@ C_I32, C_I64, C_RES_I16, C_RES_I32 = 0, 1, 2, 3
 SIDE_A, SIDE_B = 0, 1
 ROWMAJOR_RxK, ROWMAJOR_KxR = 0, 1
 MAX_PRODUCTS, MAX_PLANES = 16, 8
+STATIC_WORKSPACE_BYTES = 24 << 20
 
 EXPORTS = ["awe_create", "awe_destroy", "awe_encoding_info", "awe_encoding_lut", "awe_planes_bytes",
            "awe_workspace_bytes", "awe_host_staging_bytes", "awe_encode", "awe_gemm_planes", "awe_gemm_exact",
-           "awe_gemm_exact_host", "awe_fp4_product_raw", "awe_last_device_status", "awe_launch_count",
+           "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_fp4_product_raw", "awe_last_device_status", "awe_launch_count",
            "awe_status_string"]
 
 
@@ -72,6 +73,7 @@ def lib() -> ctypes.CDLL:
     L.awe_gemm_planes.argtypes = [vp, i32, i32, vp, vp, i64, i64, i64, vp, i32, i64, i64, vp]
     L.awe_gemm_exact.argtypes = [vp, vp, i32, vp, i32, i64, i64, i64, i32, i32, vp, i32, vp, sz, vp]
     L.awe_gemm_exact_host.argtypes = [vp, vp, i32, vp, i32, i64, i64, i64, i32, i32, vp, i32, vp, sz, vp]
+    L.awe_gemm_exact_static.argtypes = [vp, i32, vp, i32, i64, i64, i64, i32, i32, vp, i32, vp]
     L.awe_fp4_product_raw.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
     L.awe_last_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.awe_launch_count.argtypes = [vp]
@@ -197,6 +199,15 @@ def awe_gemm_exact_host(h: Handle, A_host, a_dt: int, B_host, b_dt: int, M: int,
     _check(lib().awe_gemm_exact_host(h.raw, _ptr(A_host), a_dt, _ptr(B_host), b_dt, M, N, K, enc, modulus,
                                      _ptr(C_host), out_dt, _ptr(scratch), scratch_bytes, _stream(stream)),
            "awe_gemm_exact_host")
+
+
+def awe_gemm_exact_static(A, a_dt: int, B, b_dt: int, M: int, N: int, K: int, enc: int, modulus: int, C,
+                          out_dt: int, stream=None) -> None:
+    """awe_gemm_exact for callers that must not allocate: no handle, no workspace argument; the
+    library's built-in device array (at most STATIC_WORKSPACE_BYTES of planes) is the scratch.
+    Runs on the current CUDA device; calls that could overlap on the GPU must be serialised."""
+    _check(lib().awe_gemm_exact_static(_ptr(A), a_dt, _ptr(B), b_dt, M, N, K, enc, modulus, _ptr(C), out_dt,
+                                       _stream(stream)), "awe_gemm_exact_static")
 
 
 def awe_fp4_product_raw(h: Handle, planeX, planeY, M: int, N: int, K: int, P, ldp: int, stream=None) -> None:
