@@ -31,6 +31,7 @@ if ROOT not in sys.path:
 METRIC = "effective exact INT8xINT8 TOPS (2*M*N*K / time), AWE 6-GEMM"
 NOMINAL_FP4_TFLOPS = 9000.0          # published dense FP4 peak of one B200 (paper, Section 6.2)
 NOMINAL_FP4_OVER_BF16 = 4.0          # 9.0 / 2.25 PFLOP/s nominal
+MAC_PER_CLK_PER_SM = 16384           # dense FP4: 4 x the 4096 bf16 MAC/clk/SM of the tcgen05 pipe
 
 
 def measured_peaks():
@@ -245,6 +246,7 @@ def main():
     ms_encode = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     ms_gemm = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
     assert b.awe_last_device_status(h) == (0, 0)
+    gemm_mhz = b.awe_last_gemm_clock_mhz(h)       # SM clock measured inside the last timed GEMM launch
 
     # ---- end to end from pinned host buffers through awe_gemm_exact_host
     Ah, Bh = torch.from_numpy(A).pin_memory(), torch.from_numpy(B).pin_memory()
@@ -270,8 +272,12 @@ def main():
         ms_e2e = float(t.item())
     parity_ok = parity_ok and bool(torch.equal(Ch, C.cpu()))
     clocks = sampler.stop()
+    clocks["sm_mhz_in_gemm_kernel"] = gemm_mhz
+    clocks["note"] = ("sm_mhz: NVML samples during the timed regions; sm_mhz_in_gemm_kernel: SM cycles / "
+                      "wall time measured inside the last timed GEMM launch")
 
     ops = 2.0 * M * N * K
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
     peaks = measured_peaks()
     fp4_peak = peaks["bf16_tflops_sustained"] * NOMINAL_FP4_OVER_BF16
     gemm_tflops = desc.r * ops / (ms_gemm * 1e-3) / 1e12
@@ -297,6 +303,8 @@ def main():
                      "peak_source": "%s bf16 sustained %.1f TFLOP/s x nominal fp4:bf16 ratio 4" %
                                     (peaks["source"], peaks["bf16_tflops_sustained"]),
                      "frac_of_nominal_9pflops": gemm_tflops / NOMINAL_FP4_TFLOPS,
+                     "frac_of_pipe_peak_at_delivered_clock":
+                         gemm_tflops / (MAC_PER_CLK_PER_SM * 2 * sm_count * gemm_mhz * 1e6 / 1e12) if gemm_mhz else None,
                      "frac_of_burst_peak": gemm_tflops / (peaks["bf16_tflops"] * NOMINAL_FP4_OVER_BF16)},
         "encode_roofline": {"bound": "hbm", "achieved": (M * K + K * N) * (1 + desc.n_planes_a / 2.0) / (ms_encode * 1e-3) / 1e9,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s"},

@@ -202,6 +202,12 @@ awe_status_t awe_fp4_product_raw(awe_handle_t h, const void* planeX_dev, const v
  * *site (may be NULL) naming the wait that gave up.  The word is cleared by the read. */
 awe_status_t awe_last_device_status(awe_handle_t h, void* stream, int* site);
 
+/* Diagnostic: the SM clock (MHz) at which the most recent GEMM launch on this handle actually ran,
+ * measured inside the kernel by CTA 0 as elapsed SM cycles over elapsed nanoseconds.  Waits for
+ * `stream`.  Lets a benchmark state the tensor-pipe peak at the delivered clock (the part is
+ * power-capped under FP4 load).  (No counterpart in the paper.) */
+awe_status_t awe_last_gemm_clock_mhz(awe_handle_t h, void* stream, double* mhz);
+
 /* Number of this library's kernels launched through the handle since it was created. */
 int64_t awe_launch_count(awe_handle_t h);
 

@@ -28,7 +28,7 @@ STATIC_WORKSPACE_BYTES = 24 << 20
 
 EXPORTS = ["awe_create", "awe_destroy", "awe_encoding_info", "awe_encoding_lut", "awe_planes_bytes",
            "awe_workspace_bytes", "awe_host_staging_bytes", "awe_encode", "awe_gemm_planes", "awe_gemm_exact",
-           "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_fp4_product_raw", "awe_last_device_status", "awe_launch_count",
+           "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_fp4_product_raw", "awe_last_device_status", "awe_last_gemm_clock_mhz", "awe_launch_count",
            "awe_status_string"]
 
 
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
     L.awe_gemm_exact_static.argtypes = [vp, i32, vp, i32, i64, i64, i64, i32, i32, vp, i32, vp]
     L.awe_fp4_product_raw.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
     L.awe_last_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    L.awe_last_gemm_clock_mhz.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
     L.awe_launch_count.argtypes = [vp]
     L.awe_launch_count.restype = i64
     L.awe_status_string.argtypes = [i32]
@@ -219,6 +220,12 @@ def awe_last_device_status(h: Handle, stream=None):
     site = ctypes.c_int(0)
     st = lib().awe_last_device_status(h.raw, _stream(stream), ctypes.byref(site))
     return int(st), int(site.value)
+
+
+def awe_last_gemm_clock_mhz(h: Handle, stream=None) -> float:
+    mhz = ctypes.c_double(0.0)
+    _check(lib().awe_last_gemm_clock_mhz(h.raw, _stream(stream), ctypes.byref(mhz)), "awe_last_gemm_clock_mhz")
+    return float(mhz.value)
 
 
 def awe_launch_count(h: Handle) -> int:

@@ -19,8 +19,8 @@ extern "C" awe_status_t awe_create(awe_handle_t* out, int device) {
     if (!h) return AWE_ERR_CUDA;
     h->device = device;
     h->sm_count = prop.multiProcessorCount;
-    if (cudaMalloc(&h->status_dev, 2 * sizeof(unsigned int)) != cudaSuccess ||
-        cudaMemset(h->status_dev, 0, 2 * sizeof(unsigned int)) != cudaSuccess ||
+    if (cudaMalloc(&h->status_dev, kStatusWords * sizeof(unsigned int)) != cudaSuccess ||
+        cudaMemset(h->status_dev, 0, kStatusWords * sizeof(unsigned int)) != cudaSuccess ||
         cudaMalloc(&h->lut_arena_dev, (size_t)kLutSlots * 256 * sizeof(uint64_t)) != cudaSuccess) {
         awe_destroy(h);
         return AWE_ERR_CUDA;
@@ -147,6 +147,15 @@ extern "C" awe_status_t awe_last_device_status(awe_handle_t h, void* stream, int
     if (w[0] != 0 && cudaMemset(h->status_dev, 0, sizeof(w)) != cudaSuccess) return AWE_ERR_CUDA;
     if (site) *site = (int)w[1];
     return (awe_status_t)w[0];
+}
+
+extern "C" awe_status_t awe_last_gemm_clock_mhz(awe_handle_t h, void* stream, double* mhz) {
+    if (!h || !mhz) return AWE_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return AWE_ERR_CUDA;
+    unsigned long long w[2] = {0, 0};
+    if (cudaMemcpy(w, h->status_dev + 2, sizeof(w), cudaMemcpyDeviceToHost) != cudaSuccess) return AWE_ERR_CUDA;
+    *mhz = w[1] ? (double)w[0] / (double)w[1] * 1e3 : 0.0;
+    return AWE_OK;
 }
 
 extern "C" int64_t awe_launch_count(awe_handle_t h) { return h ? h->launches : -1; }

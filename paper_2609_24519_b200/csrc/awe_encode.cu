@@ -3,9 +3,12 @@
 // written per element.
 //
 // The per-byte table holds, for raw input byte b, a 64-bit word whose byte j carries the E2M1
-// code of stored plane j in its low nibble.  Two neighbouring elements are merged with one OR
-// (the odd element shifted left by 4), which yields the packed output byte of every plane at
-// once; byte permutes then gather 4 such words into one 32-bit output word per plane.
+// code of stored plane j in its low nibble.  Two neighbouring elements (even k, odd k) are merged
+// with one shift-add per 32-bit half (the odd element moves to the high nibbles), which yields
+// the packed output byte of every plane at once; byte permutes then gather 4 such words into one
+// 32-bit output word per plane.  In shared memory every table entry is 128 bytes wide and holds
+// one copy per lane (16 copies of the 64-bit word, or 32 copies of its low half when there are at
+// most 4 planes), so a warp's data-dependent lookups never collide on a bank.
 #include <algorithm>
 
 #include "awe_internal.h"
@@ -14,23 +17,56 @@ namespace awe {
 namespace {
 
 constexpr int kEncThreads = 256;
-constexpr int kLutReplicas = 16;  // one replica per lane of a half-warp: 64-bit lookups never conflict
-constexpr size_t kLutSmemBytes = 256 * kLutReplicas * sizeof(uint64_t);
+constexpr size_t kLutSmemBytes = 256 * 128;
+#ifndef AWE_ENC_BLOCKS_PER_SM
+#define AWE_ENC_BLOCKS_PER_SM 7
+#endif
+#ifndef AWE_KXR_LANES_K
+#define AWE_KXR_LANES_K 4
+#endif
+constexpr int kKxrLanesK = AWE_KXR_LANES_K;            // lanes side by side along k
+constexpr int kKxrRows = (32 / kKxrLanesK) * 4;       // r per warp item
+constexpr int kKxrK = kKxrLanesK * 32;                // k per warp item
 
-__device__ __forceinline__ void load_lut(uint64_t* lut_s, const uint64_t* __restrict__ lut_g) {
-    for (int i = threadIdx.x; i < 256 * kLutReplicas; i += blockDim.x) lut_s[i] = lut_g[i / kLutReplicas];
+template <int NP>
+__device__ __forceinline__ void load_lut(unsigned char* lut_s, const uint64_t* __restrict__ lut_g) {
+    if (NP > 4) {
+        uint64_t* d = reinterpret_cast<uint64_t*>(lut_s);
+        for (int i = threadIdx.x; i < 256 * 16; i += blockDim.x) d[i] = lut_g[i >> 4];
+    } else {
+        uint32_t* d = reinterpret_cast<uint32_t*>(lut_s);
+        for (int i = threadIdx.x; i < 256 * 32; i += blockDim.x) d[i] = (uint32_t)lut_g[i >> 5];
+    }
     __syncthreads();
 }
 
-// Packed bytes of all planes for the element pair (b0 even k, b1 odd k).
-__device__ __forceinline__ uint64_t pair_word(const uint64_t* lut_s, int rep, uint32_t b0, uint32_t b1) {
-    return lut_s[b0 * kLutReplicas + rep] | (lut_s[b1 * kLutReplicas + rep] << 4);
+// Byte offset of this lane's private copy inside a 128-byte table entry.
+template <int NP>
+__device__ __forceinline__ uint32_t lane_slot(int lane) {
+    return NP > 4 ? (uint32_t)(lane & 15) * 8u : (uint32_t)lane * 4u;
 }
 
-// Transpose 4 pair words into one 32-bit word per plane (4 consecutive output bytes of each plane).
+// Table words (low half: planes 0-3, high half: planes 4-7) of byte number I of `word`.
+template <int NP, int I>
+__device__ __forceinline__ uint2 lookup(const unsigned char* lut_s, uint32_t slot, uint32_t word) {
+    // entry address = byte * 128; the lane slot occupies bits below 7 and is OR-ed in
+    const uint32_t shifted = I == 0 ? (word << 7) : (word >> (8 * I - 7));
+    const uint32_t off = (shifted & 0x7F80u) | slot;
+    if (NP > 4) return *reinterpret_cast<const uint2*>(lut_s + off);
+    return make_uint2(*reinterpret_cast<const uint32_t*>(lut_s + off), 0u);
+}
+
+// 8 input bytes (two 32-bit words, ascending k) -> one packed output word per plane.
 template <int NP>
-__device__ __forceinline__ void gather4(const uint64_t (&w)[4], uint32_t (&out)[NP]) {
-    const uint32_t l0 = (uint32_t)w[0], l1 = (uint32_t)w[1], l2 = (uint32_t)w[2], l3 = (uint32_t)w[3];
+__device__ __forceinline__ void encode8(const unsigned char* lut_s, uint32_t slot, uint32_t w0, uint32_t w1,
+                                        uint32_t (&out)[NP]) {
+    const uint2 e0 = lookup<NP, 0>(lut_s, slot, w0), e1 = lookup<NP, 1>(lut_s, slot, w0);
+    const uint2 e2 = lookup<NP, 2>(lut_s, slot, w0), e3 = lookup<NP, 3>(lut_s, slot, w0);
+    const uint2 e4 = lookup<NP, 0>(lut_s, slot, w1), e5 = lookup<NP, 1>(lut_s, slot, w1);
+    const uint2 e6 = lookup<NP, 2>(lut_s, slot, w1), e7 = lookup<NP, 3>(lut_s, slot, w1);
+    // pair words: byte j = packed byte (even k low nibble, odd k high nibble) of plane j
+    const uint32_t l0 = (e1.x << 4) + e0.x, l1 = (e3.x << 4) + e2.x, l2 = (e5.x << 4) + e4.x,
+                   l3 = (e7.x << 4) + e6.x;
     const uint32_t t01 = __byte_perm(l0, l1, 0x5140), t23 = __byte_perm(l2, l3, 0x5140);
     out[0] = __byte_perm(t01, t23, 0x5410);
     if (NP > 1) out[1 % NP] = __byte_perm(t01, t23, 0x7632);
@@ -40,8 +76,8 @@ __device__ __forceinline__ void gather4(const uint64_t (&w)[4], uint32_t (&out)[
         if (NP > 3) out[3 % NP] = __byte_perm(u01, u23, 0x7632);
     }
     if (NP > 4) {
-        const uint32_t h0 = (uint32_t)(w[0] >> 32), h1 = (uint32_t)(w[1] >> 32), h2 = (uint32_t)(w[2] >> 32),
-                       h3 = (uint32_t)(w[3] >> 32);
+        const uint32_t h0 = (e1.y << 4) + e0.y, h1 = (e3.y << 4) + e2.y, h2 = (e5.y << 4) + e4.y,
+                       h3 = (e7.y << 4) + e6.y;
         const uint32_t s01 = __byte_perm(h0, h1, 0x5140), s23 = __byte_perm(h2, h3, 0x5140);
         out[4 % NP] = __byte_perm(s01, s23, 0x5410);
         if (NP > 5) out[5 % NP] = __byte_perm(s01, s23, 0x7632);
@@ -53,16 +89,16 @@ __device__ __forceinline__ void gather4(const uint64_t (&w)[4], uint32_t (&out)[
     }
 }
 
-// 8 input bytes (two 32-bit words, ascending k) -> one output word per plane.
+// 32 consecutive elements of one plane row (8 words, ascending k) -> 16 packed bytes per plane.
 template <int NP>
-__device__ __forceinline__ void encode8(const uint64_t* lut_s, int rep, uint32_t lo, uint32_t hi,
-                                        uint32_t (&out)[NP]) {
-    uint64_t w[4];
-    w[0] = pair_word(lut_s, rep, lo & 0xFF, (lo >> 8) & 0xFF);
-    w[1] = pair_word(lut_s, rep, (lo >> 16) & 0xFF, lo >> 24);
-    w[2] = pair_word(lut_s, rep, hi & 0xFF, (hi >> 8) & 0xFF);
-    w[3] = pair_word(lut_s, rep, (hi >> 16) & 0xFF, hi >> 24);
-    gather4<NP>(w, out);
+__device__ __forceinline__ void encode32_store(const unsigned char* lut_s, uint32_t slot, const uint32_t (&in)[8],
+                                               uint8_t* dst, int64_t plane_stride) {
+    uint32_t o[4][NP];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) encode8<NP>(lut_s, slot, in[2 * g], in[2 * g + 1], o[g]);
+#pragma unroll
+    for (int j = 0; j < NP; ++j)
+        *reinterpret_cast<uint4*>(dst + j * plane_stride) = make_uint4(o[0][j], o[1][j], o[2][j], o[3][j]);
 }
 
 // Operand stored with the reduction index contiguous (A as M x K): a warp handles 1024
@@ -71,9 +107,10 @@ template <int NP>
 __global__ void __launch_bounds__(kEncThreads)
 encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld, const uint64_t* __restrict__ lut_g,
                   uint8_t* __restrict__ planes, int64_t pitch, int64_t plane_stride, int vec_ok) {
-    extern __shared__ __align__(16) uint64_t lut_s[];
-    load_lut(lut_s, lut_g);
-    const int lane = threadIdx.x & 31, rep = lane & (kLutReplicas - 1);
+    extern __shared__ __align__(128) unsigned char lut_s[];
+    load_lut<NP>(lut_s, lut_g);
+    const int lane = threadIdx.x & 31;
+    const uint32_t slot = lane_slot<NP>(lane);
     const int64_t Kp = pitch * 2;
     const int64_t chunks = (Kp + 1023) / 1024;
     const int64_t items = R * chunks;
@@ -101,73 +138,65 @@ encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
                 in[i] = word;
             }
         }
-        uint32_t o[4][NP];
-#pragma unroll
-        for (int g = 0; g < 4; ++g) encode8<NP>(lut_s, rep, in[2 * g], in[2 * g + 1], o[g]);
-        uint8_t* dst = planes + row * pitch + k0 / 2;
-#pragma unroll
-        for (int j = 0; j < NP; ++j)
-            *reinterpret_cast<uint4*>(dst + j * plane_stride) = make_uint4(o[0][j], o[1][j], o[2][j], o[3][j]);
+        encode32_store<NP>(lut_s, slot, in, planes + row * pitch + k0 / 2, plane_stride);
     }
 }
 
-// Operand stored with the reduction index strided (B as K x N): a block transposes a tile of
-// 128 k x 128 r through shared memory; each thread then encodes 64 consecutive k of one r.
-constexpr int kTile = 128;
-
+// Operand stored with the reduction index strided (B as K x N).  A warp handles kKxrRows
+// consecutive r by kKxrK consecutive k: kKxrLanesK neighbouring lanes own the same 4 rows and
+// consecutive runs of 32 k.  Each lane loads the 32 words X[k][r..r+3] of its k run (a warp-wide
+// load covers kKxrLanesK row segments of 128/kKxrLanesK bytes), transposes them in registers with
+// byte permutes into 4 rows of 32 consecutive k, and encodes each row exactly like the kernel
+// above.  The lanes of a group write adjacent 16-byte pieces in the same instruction, so whole
+// 32-byte sectors are written at once (a sector left half written costs a fill from DRAM).
 template <int NP>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kxr_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld, const uint64_t* __restrict__ lut_g,
                   uint8_t* __restrict__ planes, int64_t pitch, int64_t plane_stride, int vec_ok) {
-    extern __shared__ __align__(16) uint64_t smem_all[];
-    uint64_t* lut_s = smem_all;
-    uint8_t* tile = reinterpret_cast<uint8_t*>(smem_all) + kLutSmemBytes;  // [128 k][128 r]
-    load_lut(lut_s, lut_g);
-    const int t = threadIdx.x, rep = t & (kLutReplicas - 1);
+    extern __shared__ __align__(128) unsigned char lut_s[];
+    load_lut<NP>(lut_s, lut_g);
+    const int lane = threadIdx.x & 31;
+    const uint32_t slot = lane_slot<NP>(lane);
     const int64_t Kp = pitch * 2;
-    const int64_t tiles_k = Kp / kTile, tiles_r = (R + kTile - 1) / kTile;
-    for (int64_t tid = blockIdx.x; tid < tiles_k * tiles_r; tid += gridDim.x) {
-        const int64_t k0 = (tid % tiles_k) * kTile, r0 = (tid / tiles_k) * kTile;
-        if (vec_ok && r0 + kTile <= R) {
+    const int64_t k_items = (Kp + kKxrK - 1) / kKxrK, r_items = (R + kKxrRows - 1) / kKxrRows;
+    const int64_t items = k_items * r_items;
+    const int64_t warps_total = (int64_t)gridDim.x * (kEncThreads / 32);
+    for (int64_t it = (int64_t)blockIdx.x * (kEncThreads / 32) + (threadIdx.x >> 5); it < items; it += warps_total) {
+        // neighbouring warps take neighbouring r blocks of the same k range: their loads share k rows
+        const int64_t r0 = (it % r_items) * kKxrRows + (lane / kKxrLanesK) * 4;
+        const int64_t k0 = (it / r_items) * kKxrK + (lane % kKxrLanesK) * 32;
+        if (r0 >= R || k0 >= Kp) continue;
+        uint32_t raw[32];  // raw[i] = bytes X[k0+i][r0..r0+3]
+        if (vec_ok && r0 + 4 <= R && k0 + 32 <= K) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = i * 32 + (t >> 3), c16 = t & 7;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (k0 + row < K) v = __ldg(reinterpret_cast<const uint4*>(X + (k0 + row) * ld + r0) + c16);
-                *reinterpret_cast<uint4*>(tile + row * kTile + c16 * 16) = v;
-            }
+            for (int i = 0; i < 32; ++i) raw[i] = __ldg(reinterpret_cast<const uint32_t*>(X + (k0 + i) * ld + r0));
         } else {
-            for (int i = 0; i < kTile * kTile / kEncThreads; ++i) {
-                const int idx = i * kEncThreads + t, row = idx / kTile, col = idx % kTile;
-                int8_t v = 0;
-                if (k0 + row < K && r0 + col < R) v = X[(k0 + row) * ld + r0 + col];
-                tile[row * kTile + col] = (uint8_t)v;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                uint32_t word = 0;
+                if (k0 + i < K) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (r0 + j < R) word |= (uint32_t)(uint8_t)X[(k0 + i) * ld + r0 + j] << (8 * j);
+                }
+                raw[i] = word;
             }
         }
-        __syncthreads();
-        const int rl = t & (kTile - 1), kh = t >> 7;
-        const int64_t r = r0 + rl;
-        uint32_t o[8][NP];
+        // 4x4 byte transposes: t[j][g] = the 4 bytes of row r0+j at k0+4g .. k0+4g+3
+        uint32_t t[4][8];
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
-            uint32_t lo = 0, hi = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                lo |= (uint32_t)tile[(kh * 64 + g * 8 + j) * kTile + rl] << (8 * j);
-                hi |= (uint32_t)tile[(kh * 64 + g * 8 + 4 + j) * kTile + rl] << (8 * j);
-            }
-            encode8<NP>(lut_s, rep, lo, hi, o[g]);
+            const uint32_t a = raw[4 * g], b = raw[4 * g + 1], c = raw[4 * g + 2], d = raw[4 * g + 3];
+            const uint32_t ab_lo = __byte_perm(a, b, 0x5140), cd_lo = __byte_perm(c, d, 0x5140);
+            const uint32_t ab_hi = __byte_perm(a, b, 0x7362), cd_hi = __byte_perm(c, d, 0x7362);
+            t[0][g] = __byte_perm(ab_lo, cd_lo, 0x5410);
+            t[1][g] = __byte_perm(ab_lo, cd_lo, 0x7632);
+            t[2][g] = __byte_perm(ab_hi, cd_hi, 0x5410);
+            t[3][g] = __byte_perm(ab_hi, cd_hi, 0x7632);
         }
-        if (r < R) {
-            uint8_t* dst = planes + r * pitch + (k0 + kh * 64) / 2;
 #pragma unroll
-            for (int j = 0; j < NP; ++j) {
-                uint4* d = reinterpret_cast<uint4*>(dst + j * plane_stride);
-                d[0] = make_uint4(o[0][j], o[1][j], o[2][j], o[3][j]);
-                d[1] = make_uint4(o[4][j], o[5][j], o[6][j], o[7][j]);
-            }
-        }
-        __syncthreads();
+        for (int j = 0; j < 4; ++j)
+            if (r0 + j < R) encode32_store<NP>(lut_s, slot, t[j], planes + (r0 + j) * pitch + k0 / 2, plane_stride);
     }
 }
 
@@ -175,24 +204,17 @@ template <int NP>
 cudaError_t launch(awe_layout_t layout, const int8_t* X, int64_t R, int64_t K, int64_t ld, const uint64_t* lut,
                    uint8_t* planes, int64_t pitch, int64_t plane_stride, int vec_ok, int sm_count,
                    cudaStream_t stream) {
+    const int64_t warps_per_block = kEncThreads / 32;
     if (layout == AWE_ROWMAJOR_RxK) {
         const int64_t items = R * ((pitch * 2 + 1023) / 1024);
-        const int64_t blocks = std::min<int64_t>((items + 7) / 8, (int64_t)sm_count * 4);
+        const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
         encode_rxk_kernel<NP><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(X, R, K, ld, lut, planes,
                                                                                         pitch, plane_stride, vec_ok);
     } else {
-        const size_t smem = kLutSmemBytes + kTile * kTile;
-        static bool attr_set[AWE_MAX_PLANES + 1] = {false};
-        if (!attr_set[NP]) {
-            cudaError_t e = cudaFuncSetAttribute(encode_kxr_kernel<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 (int)smem);
-            if (e != cudaSuccess) return e;
-            attr_set[NP] = true;
-        }
-        const int64_t tiles = (pitch * 2 / kTile) * ((R + kTile - 1) / kTile);
-        const int64_t blocks = std::min<int64_t>(tiles, (int64_t)sm_count * 4);
-        encode_kxr_kernel<NP><<<(unsigned)blocks, kEncThreads, smem, stream>>>(X, R, K, ld, lut, planes, pitch,
-                                                                              plane_stride, vec_ok);
+        const int64_t items = ((pitch * 2 + kKxrK - 1) / kKxrK) * ((R + kKxrRows - 1) / kKxrRows);
+        const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
+        encode_kxr_kernel<NP><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(X, R, K, ld, lut, planes,
+                                                                                        pitch, plane_stride, vec_ok);
     }
     return cudaGetLastError();
 }
@@ -218,7 +240,9 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
     awe_status_t s = device_lut(h, enc, modulus, side, dt, st, &lut);
     if (s != AWE_OK) return s;
     const int64_t pitch = plane_pitch_bytes(K), plane_stride = R * pitch;
-    const int vec_ok = ((uintptr_t)X_dev % 16 == 0) && (ld % 16 == 0);
+    // vector path: 16-byte loads along k (RxK) or 4-byte loads along r (KxR)
+    const int64_t align = layout == AWE_ROWMAJOR_RxK ? 16 : 4;
+    const int vec_ok = ((uintptr_t)X_dev % align == 0) && (ld % align == 0);
     const int8_t* X = (const int8_t*)X_dev;
     uint8_t* P = (uint8_t*)planes_dev;
     cudaError_t e;

@@ -54,9 +54,14 @@ constexpr int kMaxStages = 6;
 constexpr int kThreads = 320;
 constexpr int kEpiWarps = 8;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kAccCol = 0;
-constexpr uint32_t kSfaCol = 256;  // 16 columns of constant scale bytes each for A and B
-constexpr uint32_t kSfbCol = 272;
+// Two accumulators of 256 columns and 32 columns of scale bytes do not fit 512 columns side by
+// side, so accumulator 1 starts inside the last 32 columns of accumulator 0.  The epilogue reads
+// those shared columns first and releases them separately (overlap_free), which lets the MMAs of
+// the next segment start while the rest of the previous accumulator is still being drained.
+constexpr uint32_t kAccCol0 = 0;
+constexpr uint32_t kAccCol1 = 224;
+constexpr uint32_t kSfaCol = 480;  // 16 columns of constant scale bytes each for A and B
+constexpr uint32_t kSfbCol = 496;
 
 enum OutMode { OUT_I32 = 0, OUT_I64 = 1, OUT_RES_I16 = 2, OUT_RES_I32 = 3, OUT_RAW_F32 = 4 };
 
@@ -73,6 +78,7 @@ struct GemmParams {
     void* C;
     long long ldc;
     unsigned int* status;
+    unsigned long long* clock_probe;  // [0] SM cycles, [1] nanoseconds spent by CTA 0 in this launch
     int vec_store;     // C rows are 16-byte aligned: vector stores allowed
     float acc_scale;   // accumulator value -> product of doubled integers
     uint32_t sf_word;  // four copies of the UE8M0 scale byte
@@ -81,8 +87,9 @@ struct GemmParams {
 struct Shared {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
-    uint64_t tmem_full;
-    uint64_t tmem_empty;
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint64_t overlap_free;
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
 };
@@ -124,6 +131,44 @@ __device__ __forceinline__ int fast_mod(int x, int m, float inv_m) {
     return r;
 }
 
+struct EpiMath {
+    int out_mode, m;
+    float inv_m, acc_scale;
+};
+
+// All lanes of the warp have finished reading their TMEM columns: one arrival for the warp on a
+// barrier of this CTA or, in a pair, of CTA 0 (cluster address).
+__device__ __forceinline__ void release(uint32_t bar, int lane, bool remote) {
+    ptx::tc_fence_before();
+    __syncwarp();
+    if (lane == 0) {
+        if (remote) ptx::mbar_arrive_cluster(bar);
+        else ptx::mbar_arrive(bar);
+    }
+}
+
+// Drain 32 accumulator columns (block BLK of this thread's 128) and fold them into the running sums.
+template <int BLK>
+__device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128], const EpiMath& em, int ell) {
+    uint32_t v[32];
+    ptx::tmem_ld_32x32(taddr + BLK * 32, v);
+    ptx::tmem_wait_ld();
+    if (em.out_mode == OUT_RAW_F32) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) sum[BLK * 32 + i] = __float_as_uint(__uint_as_float(v[i]) * em.acc_scale);
+    } else if (em.m) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int pm = fast_mod(__float2int_rn(__uint_as_float(v[i]) * em.acc_scale), em.m, em.inv_m);
+            sum[BLK * 32 + i] = (uint32_t)fast_mod((int)sum[BLK * 32 + i] + ell * pm, em.m, em.inv_m);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            sum[BLK * 32 + i] += (uint32_t)ell * (uint32_t)__float2int_rn(__uint_as_float(v[i]) * em.acc_scale);
+    }
+}
+
 template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -147,8 +192,11 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
         }
-        ptx::mbar_init(ptx::smem_u32(&sh->tmem_full), 1);
-        ptx::mbar_init(ptx::smem_u32(&sh->tmem_empty), kEpiWarps * C::kCtas);
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(ptx::smem_u32(&sh->acc_full[b]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh->acc_empty[b]), kEpiWarps * C::kCtas);
+        }
+        ptx::mbar_init(ptx::smem_u32(&sh->overlap_free), (kEpiWarps / 2) * C::kCtas);
         sh->abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&map_a);
@@ -180,6 +228,13 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
+
+    // CTA 0 measures the SM clock it actually ran at (cycles over wall time of the launch)
+    unsigned long long probe_c0 = 0, probe_t0 = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        probe_c0 = clock64();
+        probe_t0 = ptx::globaltimer_ns();
+    }
 
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int chunks = (p.num_kblocks + p.chunk_kblocks - 1) / p.chunk_kblocks;
@@ -224,7 +279,15 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             for (int t = worker; t < num_tiles && ok; t += num_workers) {
                 for (int k = 0; k < p.r && ok; ++k) {
                     for (int c = 0; c < chunks && ok; ++c, ++drains) {
-                        if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->tmem_empty), (drains & 1u) ^ 1u, p.status, 2)))
+                        // accumulator (drains & 1): its previous contents (two segments ago) fully drained,
+                        // and the columns it shares with the other accumulator already read
+                        const uint32_t ab = drains & 1u;
+                        const uint32_t acc_col = ab ? kAccCol1 : kAccCol0;
+                        if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->acc_empty[ab]), ((drains >> 1) & 1u) ^ 1u,
+                                                p.status, 2)))
+                            break;
+                        if (drains > 0 &&
+                            !(ok = bounded_wait(sh, ptx::smem_u32(&sh->overlap_free), (drains - 1u) & 1u, p.status, 5)))
                             break;
                         ptx::tc_fence_after();
                         const int kb_end = min(p.num_kblocks, (c + 1) * p.chunk_kblocks);
@@ -240,10 +303,10 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                                 // 64 elements = 32 bytes further along K inside the swizzle row
                                 const uint32_t acc = (kb > c * p.chunk_kblocks || j > 0) ? 1u : 0u;
                                 if (kPair)
-                                    ptx::mma_mxf4_pair(tmem + kAccCol, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
+                                    ptx::mma_mxf4_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
                                                        tmem + kSfaCol, tmem + kSfbCol, acc);
                                 else
-                                    ptx::mma_mxf4(tmem + kAccCol, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
+                                    ptx::mma_mxf4(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
                                                   tmem + kSfaCol, tmem + kSfbCol, acc);
                             }
                             // frees the stage in both CTAs of a pair
@@ -251,8 +314,8 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             else ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));
                         }
                         if (ok) {
-                            if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->tmem_full), 3);
-                            else ptx::mma_commit(ptx::smem_u32(&sh->tmem_full));
+                            if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->acc_full[ab]), 3);
+                            else ptx::mma_commit(ptx::smem_u32(&sh->acc_full[ab]));
                         }
                     }
                 }
@@ -261,13 +324,19 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     } else {
         // -------------------------------------------------------------------- epilogue
         const int quarter = warp & 3, half = (warp - 2) >> 2;
-        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + kAccCol + (uint32_t)half * 128u;
+        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)half * 128u;
         const int m = p.modulus;
         const float inv_m = m ? 1.0f / (float)m : 0.0f;
         uint32_t drains = 0;
         bool ok = true;
-        const uint32_t tmem_empty_bar = kPair ? ptx::map_to_cta(ptx::smem_u32(&sh->tmem_empty), 0)
-                                              : ptx::smem_u32(&sh->tmem_empty);
+        // barriers the MMA issuer (CTA 0) waits on
+        uint32_t acc_empty_bar[2], overlap_bar = ptx::smem_u32(&sh->overlap_free);
+        for (int b = 0; b < 2; ++b) acc_empty_bar[b] = ptx::smem_u32(&sh->acc_empty[b]);
+        if (kPair) {
+            overlap_bar = ptx::map_to_cta(overlap_bar, 0);
+            for (int b = 0; b < 2; ++b) acc_empty_bar[b] = ptx::map_to_cta(acc_empty_bar[b], 0);
+        }
+        const EpiMath em = {p.out_mode, m, inv_m, p.acc_scale};
         for (int t = worker; t < num_tiles && ok; t += num_workers) {
             int tm, tn;
             tile_coords(t, p.tiles_m, p.tiles_n, &tm, &tn);
@@ -277,34 +346,28 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             for (int k = 0; k < p.r && ok; ++k) {
                 const int ell = p.ell[k];
                 for (int c = 0; c < chunks && ok; ++c, ++drains) {
-                    ok = bounded_wait(sh, ptx::smem_u32(&sh->tmem_full), drains & 1u, p.status, 4);
+                    const uint32_t ab = drains & 1u;
+                    ok = bounded_wait(sh, ptx::smem_u32(&sh->acc_full[ab]), (drains >> 1) & 1u, p.status, 4);
                     ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below need the whole warp
                     if (!ok) break;
                     ptx::tc_fence_after();
-#pragma unroll
-                    for (int b = 0; b < 4; ++b) {
-                        uint32_t v[32];
-                        ptx::tmem_ld_32x32(taddr + b * 32, v);
-                        ptx::tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const float f = __uint_as_float(v[i]) * p.acc_scale;
-                            if (p.out_mode == OUT_RAW_F32) {
-                                sum[b * 32 + i] = __float_as_uint(f);
-                            } else if (m) {
-                                const int pm = fast_mod(__float2int_rn(f), m, inv_m);
-                                sum[b * 32 + i] = (uint32_t)fast_mod((int)sum[b * 32 + i] + ell * pm, m, inv_m);
-                            } else {
-                                sum[b * 32 + i] += (uint32_t)ell * (uint32_t)__float2int_rn(f);
-                            }
-                        }
+                    // The 32 columns shared by the two accumulators are the last block of accumulator 0
+                    // (held by the warps of column half 1) and the first block of accumulator 1 (half 0):
+                    // they are read first and handed back at once.
+                    if (ab == 0) {
+                        drain_block<3>(taddr + kAccCol0, sum, em, ell);
+                        if (half == 1) release(overlap_bar, lane, kPair);
+                        drain_block<0>(taddr + kAccCol0, sum, em, ell);
+                        drain_block<1>(taddr + kAccCol0, sum, em, ell);
+                        drain_block<2>(taddr + kAccCol0, sum, em, ell);
+                    } else {
+                        drain_block<0>(taddr + kAccCol1, sum, em, ell);
+                        if (half == 0) release(overlap_bar, lane, kPair);
+                        drain_block<1>(taddr + kAccCol1, sum, em, ell);
+                        drain_block<2>(taddr + kAccCol1, sum, em, ell);
+                        drain_block<3>(taddr + kAccCol1, sum, em, ell);
                     }
-                    ptx::tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (kPair) ptx::mbar_arrive_cluster(tmem_empty_bar);
-                        else ptx::mbar_arrive(tmem_empty_bar);
-                    }
+                    release(acc_empty_bar[ab], lane, kPair);
                 }
             }
             if (!ok) break;
@@ -384,6 +447,10 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0 && p.clock_probe) {
+        p.clock_probe[0] = clock64() - probe_c0;
+        p.clock_probe[1] = ptx::globaltimer_ns() - probe_t0;
+    }
     if (kPair) ptx::cluster_sync_all();  // neither CTA leaves while the other may still signal it
     if (warp == 1) {
         ptx::tc_fence_after();
@@ -434,6 +501,7 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
     p.tiles_m = (p.M + kTileM * C::kCtas - 1) / (kTileM * C::kCtas);
     p.tiles_n = (p.N + kTileN - 1) / kTileN;
     p.status = h->status_dev;
+    p.clock_probe = reinterpret_cast<unsigned long long*>(h->status_dev + 2);
     const int workers = std::min(p.tiles_m * p.tiles_n, h->sm_count / C::kCtas);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(workers * C::kCtas));

@@ -48,7 +48,7 @@ inline int64_t plane_pitch_bytes(int64_t K) { return round_up(K, 256) / 2; }
 struct awe_ctx {
     int device = 0;
     int sm_count = 0;
-    unsigned int* status_dev = nullptr;  // [0] = status, [1] = site
+    unsigned int* status_dev = nullptr;  // [0] = status, [1] = site, [2..5] = clock probe of the last GEMM launch
     uint64_t* lut_arena_dev = nullptr;   // kLutSlots tables of 256 x u64
     struct LutSlot {
         int enc, modulus, side, dt;
@@ -61,6 +61,7 @@ struct awe_ctx {
 
 namespace awe {
 constexpr int kLutSlots = 96;
+constexpr int kStatusWords = 8;
 // Device pointer of the 256-entry u64 table for (enc, modulus, side, dt); uploads on first use.
 awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_in_dtype_t dt,
                         cudaStream_t stream, const uint64_t** out);
