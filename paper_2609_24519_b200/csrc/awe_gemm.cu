@@ -37,20 +37,23 @@ constexpr int kTileN = 256;
 constexpr int kBlockKBytes = 128;  // 256 E2M1 elements: one 128-byte swizzle row
 constexpr int kABytes = kTileM * kBlockKBytes;  // 16 KB
 
+#ifndef AWE_PAIR_STAGES
+#define AWE_PAIR_STAGES 6
+#endif
 // Per-variant sizes: a CTA of a pair stages only half of the B tile.
 template <bool kPair>
 struct Cfg {
     static constexpr int kBRows = kPair ? kTileN / 2 : kTileN;
     static constexpr int kBBytes = kBRows * kBlockKBytes;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kStages = kPair ? 6 : 4;
+    static constexpr int kStages = kPair ? AWE_PAIR_STAGES : 4;
     static constexpr int kCtas = kPair ? 2 : 1;
     static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
     // mxf4 instruction descriptor: E2M1 x E2M1, both K-major, UE8M0 scales, dense K = 64
     static constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | (1u << 23) |
                                        ((uint32_t)((kTileM * kCtas) >> 4) << 24);
 };
-constexpr int kMaxStages = 6;
+constexpr int kMaxStages = 7;
 constexpr int kThreads = 320;
 constexpr int kEpiWarps = 8;
 constexpr uint32_t kTmemCols = 512;
