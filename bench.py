@@ -31,6 +31,7 @@ if ROOT not in sys.path:
 METRIC = "effective exact INT8xINT8 TOPS (2*M*N*K / time), AWE 6-GEMM"
 NOMINAL_FP4_TFLOPS = 9000.0          # published dense FP4 peak of one B200 (paper, Section 6.2)
 NOMINAL_FP4_OVER_BF16 = 4.0          # 9.0 / 2.25 PFLOP/s nominal
+GEMM_DRAM_BYTES_8192 = 1524829696 + 262142208   # ncu capture of awe_gemm_kernel at 8192^3, AWE-6
 MAC_PER_CLK_PER_SM = 16384           # dense FP4: 4 x the 4096 bf16 MAC/clk/SM of the tcgen05 pipe
 
 
@@ -179,10 +180,10 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
+    from paper_2609_24519_b200 import replicas
+
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(dev)
 
     h = b.awe_create(local_rank)
     enc, M, N, K = b.ENC_INT8_AWE6, w.M, w.N, w.K
@@ -237,11 +238,8 @@ def main():
     barrier()
     sampler.region(False)
     launches = b.awe_launch_count(h) - launches0
-    ms_total = t_start.elapsed_time(t_end)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ops = 2.0 * M * N * K
+    ms_total, ops_all_ranks = replicas.aggregate(t_start.elapsed_time(t_end), ops * args.steps, dev)
     ms_step = ms_total / args.steps
     ms_encode = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     ms_gemm = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
@@ -265,24 +263,20 @@ def main():
     e1.record()
     barrier()
     sampler.region(False)
-    ms_e2e = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    ms_e2e_total, ops_e2e_all = replicas.aggregate(e0.elapsed_time(e1), ops * e2e_steps, dev)
+    ms_e2e = ms_e2e_total / e2e_steps
     parity_ok = parity_ok and bool(torch.equal(Ch, C.cpu()))
     clocks = sampler.stop()
     clocks["sm_mhz_in_gemm_kernel"] = gemm_mhz
     clocks["note"] = ("sm_mhz: NVML samples during the timed regions; sm_mhz_in_gemm_kernel: SM cycles / "
                       "wall time measured inside the last timed GEMM launch")
 
-    ops = 2.0 * M * N * K
     sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
     peaks = measured_peaks()
     fp4_peak = peaks["bf16_tflops_sustained"] * NOMINAL_FP4_OVER_BF16
     gemm_tflops = desc.r * ops / (ms_gemm * 1e-3) / 1e12
     line = {
-        "metric": METRIC, "value": world * ops / (ms_step * 1e-3) / 1e12, "unit": "TOPS", "n_gpus": world,
+        "metric": METRIC, "value": ops_all_ranks / (ms_total * 1e-3) / 1e12, "unit": "TOPS", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "e2m1 (fp4) operands, f32 accumulate, int32 reconstruction",
         "data": "synthetic",
@@ -291,14 +285,16 @@ def main():
                    "l2": "no flush: per-step working set (64+64 MiB in, 384 MiB planes, 256 MiB out) exceeds the 126 MB L2",
                    "parallelism": "replicas only (no exchange step)" if world > 1 else "single GPU"},
         "clocks": clocks,
-        "e2e": {"value": world * ops / (ms_e2e * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms_e2e,
+        "e2e": {"value": ops_e2e_all / (ms_e2e_total * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms_e2e,
                 "steps": e2e_steps, "h2d_bytes_per_step": int(A.nbytes + B.nbytes), "d2h_bytes_per_step": int(M * N * 4)},
         "gpu_launches": int(launches),
         "parity": "bit-exact vs CPU oracle on %d sampled rows; 3-call path == awe_gemm_exact == host path" % len(rows)
                   if parity_ok else "MISMATCH",
         "kernels_ms": {"encode_a_plus_b": ms_encode, "gemm_and_reconstruction": ms_gemm},
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
-                     "frac": gemm_tflops / fp4_peak, "traffic": None,
+                     "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_BYTES_8192 if (M, N, K) == (8192, 8192, 8192) else None,
+                     "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one launch at this workload "
+                                     "(ncu, one-pass metrics; profiles/launch_list_bench_8192_awe6.md)",
                      "kernel": "awe_gemm_kernel", "flops_per_launch": desc.r * ops,
                      "peak_source": "%s bf16 sustained %.1f TFLOP/s x nominal fp4:bf16 ratio 4" %
                                     (peaks["source"], peaks["bf16_tflops_sustained"]),
@@ -345,6 +341,46 @@ def main():
         except Exception as ex:  # library reference point only
             ctx["int8_tensor_core_gemm_TOPS"] = None
             ctx["int8_gemm_error"] = str(ex)[:100]
+        # the other configurations, device-timed through awe_gemm_exact (context only; their parity is
+        # covered by the GPU tests).  Inputs are drawn on the device from a seeded torch generator.
+        if (M, N, K) == (8192, 8192, 8192):
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(7)
+
+            def timed(enc_, mod_, a_, a_dt_, b_, out_dt_, tdt_, m_, n_, k_, iters=5):
+                ws_ = torch.empty(b.awe_workspace_bytes(enc_, mod_, m_, n_, k_), dtype=torch.uint8, device=dev)
+                c_ = torch.empty((m_, n_), dtype=tdt_, device=dev)
+                for _ in range(2):
+                    b.awe_gemm_exact(h, a_, a_dt_, b_, b.I8, m_, n_, k_, enc_, mod_, c_, out_dt_, ws_)
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(iters):
+                    b.awe_gemm_exact(h, a_, a_dt_, b_, b.I8, m_, n_, k_, enc_, mod_, c_, out_dt_, ws_)
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / iters
+
+            a4 = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device=dev, generator=gen)
+            ms = timed(b.ENC_INT4xINT8_AWE4, 0, a4, b.I4_IN_I8, dB, b.C_I32, torch.int32, 8192, 8192, 8192)
+            ctx["int4xint8_awe4_8192_TOPS"] = ops / (ms * 1e-3) / 1e12
+            del a4
+            ax = torch.randint(0, 2, (4096, 16384), dtype=torch.int8, device=dev, generator=gen) * 255 - 128
+            bx = torch.randint(0, 2, (16384, 4096), dtype=torch.int8, device=dev, generator=gen) * 255 - 128
+            ms = timed(b.ENC_INT8_AWE6, 0, ax.to(torch.int8), b.I8, bx.to(torch.int8), b.C_I64, torch.int64, 4096, 4096,
+                       16384)
+            ctx["worst_case_4096x4096x16384_int64_TOPS"] = 2.0 * 4096 * 4096 * 16384 / (ms * 1e-3) / 1e12
+            del ax, bx
+            from oracle.rns import RNS_SET_FP64   # the list of moduli only (a constant, no arithmetic)
+            total_ms, prods = 0.0, 0
+            for m_ in RNS_SET_FP64:
+                lo = -(m_ // 2)
+                am = torch.randint(lo, lo + m_, (8192, 8192), dtype=torch.int8, device=dev, generator=gen)
+                bm = torch.randint(lo, lo + m_, (8192, 8192), dtype=torch.int8, device=dev, generator=gen)
+                total_ms += timed(b.ENC_MOD_M, m_, am, b.I8, bm, b.C_RES_I16, torch.int16, 8192, 8192, 8192, iters=2)
+                prods += b.awe_encoding_info(b.ENC_MOD_M, m_).r
+                del am, bm
+            ctx["residue_22_moduli_8192_total_ms"] = total_ms
+            ctx["residue_22_moduli_fp4_gemms"] = prods
         ctx["paper_theoretical_TOPS"] = "1500 (9.0 PFLOPS / 6, published peak, not a measurement; B200)"
         line["context"] = ctx
 

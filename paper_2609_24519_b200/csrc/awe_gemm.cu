@@ -125,6 +125,11 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
     *tn = in_group / gsize;
 }
 
+// Order of the products inside a tile: ascending on a worker's even tiles, descending on its odd
+// ones, so the planes used last by one tile are the first the next tile asks L2 for.  The sum of
+// the products does not depend on the order.
+__device__ __forceinline__ int product_at(int kk, int tile_iter, int r) { return (tile_iter & 1) ? r - 1 - kk : kk; }
+
 __device__ __forceinline__ int fast_mod(int x, int m, float inv_m) {
     int q = __float2int_rz(__int2float_rn(x) * inv_m);
     int r = x - q * m;
@@ -247,12 +252,13 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // ---------------------------------------------------------------- TMA producer
             uint32_t it = 0;
             bool ok = true;
-            for (int t = worker; t < num_tiles && ok; t += num_workers) {
+            for (int t = worker, tile_iter = 0; t < num_tiles && ok; t += num_workers, ++tile_iter) {
                 int tm, tn;
                 tile_coords(t, p.tiles_m, p.tiles_n, &tm, &tn);
                 const int row_a = (tm * C::kCtas + (int)rank) * kTileM;
                 const int row_b = tn * kTileN + (int)rank * C::kBRows;
-                for (int k = 0; k < p.r && ok; ++k) {
+                for (int kk = 0; kk < p.r && ok; ++kk) {
+                    const int k = product_at(kk, tile_iter, p.r);
                     for (int kb = 0; kb < p.num_kblocks; ++kb, ++it) {
                         const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
                         if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->empty[s]), ph ^ 1u, p.status, 1))) break;
@@ -340,14 +346,14 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             for (int b = 0; b < 2; ++b) acc_empty_bar[b] = ptx::map_to_cta(acc_empty_bar[b], 0);
         }
         const EpiMath em = {p.out_mode, m, inv_m, p.acc_scale};
-        for (int t = worker; t < num_tiles && ok; t += num_workers) {
+        for (int t = worker, tile_iter = 0; t < num_tiles && ok; t += num_workers, ++tile_iter) {
             int tm, tn;
             tile_coords(t, p.tiles_m, p.tiles_n, &tm, &tn);
             uint32_t sum[128];
 #pragma unroll
             for (int i = 0; i < 128; ++i) sum[i] = 0;
-            for (int k = 0; k < p.r && ok; ++k) {
-                const int ell = p.ell[k];
+            for (int kk = 0; kk < p.r && ok; ++kk) {
+                const int ell = p.ell[product_at(kk, tile_iter, p.r)];
                 for (int c = 0; c < chunks && ok; ++c, ++drains) {
                     const uint32_t ab = drains & 1u;
                     ok = bounded_wait(sh, ptx::smem_u32(&sh->acc_full[ab]), (drains >> 1) & 1u, p.status, 4);
