@@ -57,12 +57,15 @@ typedef enum {
     AWE_ENC_INT8_BASE13_9 = 2,  /* INT8xINT8, 9 products, weights (1,13,169)  (prior work, Section 1)  */
     AWE_ENC_INT4xINT8_AWE4 = 3, /* INT4xINT8, 4 products, D = 2               (Appendix A)             */
     AWE_ENC_MOD_M = 4,          /* residue form mod `modulus`, 1/3/4 products (Section 5.3)            */
-    AWE_ENC_INT8_AWE6_ALT = 5   /* INT8xINT8, 6 products, w = v = (1,11,39)   (Section 4.3)            */
+    AWE_ENC_INT8_AWE6_ALT = 5,  /* INT8xINT8, 6 products, w = v = (1,11,39)   (Section 4.3)            */
+    AWE_ENC_TERNARY_INT8_3 = 6  /* {0,+-1}xINT8, 3 products: one limb against the three base-13 limbs
+                                   (Section 6.2), K* = 2,097,152                                       */
 } awe_encoding_t;
 
 typedef enum {
     AWE_I8 = 0,      /* one signed 8-bit value per byte                                          */
-    AWE_I4_IN_I8 = 1 /* one signed 4-bit value per byte; only the low nibble is read (sign-extended) */
+    AWE_I4_IN_I8 = 1, /* one signed 4-bit value per byte; only the low nibble is read (sign-extended) */
+    AWE_T2_IN_I8 = 2  /* one ternary value -1, 0 or +1 per byte; any other byte is read as 0         */
 } awe_in_dtype_t;
 
 typedef enum {

@@ -24,6 +24,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstdio>
 #include <cstdlib>
 
 #include "awe_internal.h"
@@ -48,7 +49,7 @@ struct Cfg {
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kStages = kPair ? AWE_PAIR_STAGES : 4;
     static constexpr int kCtas = kPair ? 2 : 1;
-    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 8 * 4096 + 256;
     // mxf4 instruction descriptor: E2M1 x E2M1, both K-major, UE8M0 scales, dense K = 64
     static constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | (1u << 23) |
                                        ((uint32_t)((kTileM * kCtas) >> 4) << 24);
@@ -56,6 +57,7 @@ struct Cfg {
 constexpr int kMaxStages = 7;
 constexpr int kThreads = 320;
 constexpr int kEpiWarps = 8;
+constexpr int kStageWarpBytes = 4096;  // 32 rows x 128 bytes per epilogue warp for the write-out
 constexpr uint32_t kTmemCols = 512;
 // Two accumulators of 256 columns and 32 columns of scale bytes do not fit 512 columns side by
 // side, so accumulator 1 starts inside the last 32 columns of accumulator 0.  The epilogue reads
@@ -130,18 +132,24 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
 // the products does not depend on the order.
 __device__ __forceinline__ int product_at(int kk, int tile_iter, int r) { return (tile_iter & 1) ? r - 1 - kk : kk; }
 
-__device__ __forceinline__ int fast_mod(int x, int m, float inv_m) {
-    int q = __float2int_rz(__int2float_rn(x) * inv_m);
-    int r = x - q * m;
-    if (r < 0) r += m;
-    if (r >= m) r -= m;
-    if (r < 0) r += m;
+// Residue arithmetic in FP32 (Section 5.3).  Every quantity is an integer of magnitude below 2^22
+// held exactly in a float; x mod m is taken without leaving the FP32 pipe: q = round(x / m) by the
+// add-and-subtract-1.5*2^23 trick, r = x - q m by one exact FMA, and one correction step in each
+// direction puts r into the symmetric range [lo, hi] = [-floor(m/2), ceil(m/2) - 1].
+__device__ __forceinline__ float mod_symmetric(float x, float m, float inv_m, float lo, float hi) {
+    const float magic = 12582912.0f;
+    const float q = __fadd_rn(__fadd_rn(__fmul_rn(x, inv_m), magic), -magic);
+    float r = __fmaf_rn(-q, m, x);
+    r = r > hi ? r - m : r;
+    r = r < lo ? r + m : r;
     return r;
 }
 
 struct EpiMath {
     int out_mode, m;
-    float inv_m, acc_scale;
+    float acc_scale;
+    float mf, inv_m, lo, hi;  // modulus and its symmetric range as floats
+    int reduce_each;          // reduce the running residue sum after every segment (very long K only)
 };
 
 // All lanes of the warp have finished reading their TMEM columns: one arrival for the warp on a
@@ -156,25 +164,90 @@ __device__ __forceinline__ void release(uint32_t bar, int lane, bool remote) {
 }
 
 // Drain 32 accumulator columns (block BLK of this thread's 128) and fold them into the running sums.
+// When `early_bar` is non-zero these are the columns the two accumulators share: they are handed
+// back to the MMA issuer as soon as they sit in registers, before any arithmetic.
 template <int BLK>
-__device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128], const EpiMath& em, int ell) {
+__device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128], const EpiMath& em, int ell,
+                                            uint32_t early_bar = 0, int lane = 0, bool remote = false) {
     uint32_t v[32];
     ptx::tmem_ld_32x32(taddr + BLK * 32, v);
     ptx::tmem_wait_ld();
+    if (early_bar) release(early_bar, lane, remote);
     if (em.out_mode == OUT_RAW_F32) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) sum[BLK * 32 + i] = __float_as_uint(__uint_as_float(v[i]) * em.acc_scale);
     } else if (em.m) {
+        // Running sum kept as a float (exact: |ell| <= m/2, |residue| <= m/2 + 1, few terms).  The
+        // accumulator holds P / acc_scale; the scale (a power of two) is folded into the constants:
+        // q = round(P / m), residue / acc_scale = acc - q (m / acc_scale), sum += (ell acc_scale) * that.
+        // No range correction here: a residue one step outside [-m/2, m/2] is still congruent.
+        const float magic = 12582912.0f;
+        const float q_scale = em.acc_scale * em.inv_m, m_scaled = em.mf / em.acc_scale;
+        const float lam = (float)ell * em.acc_scale;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-            const int pm = fast_mod(__float2int_rn(__uint_as_float(v[i]) * em.acc_scale), em.m, em.inv_m);
-            sum[BLK * 32 + i] = (uint32_t)fast_mod((int)sum[BLK * 32 + i] + ell * pm, em.m, em.inv_m);
+            const float a = __uint_as_float(v[i]);
+            const float q = __fadd_rn(__fadd_rn(__fmul_rn(a, q_scale), magic), -magic);
+            const float res = __fmaf_rn(-q, m_scaled, a);
+            float sf = __fmaf_rn(lam, res, __uint_as_float(sum[BLK * 32 + i]));
+            if (em.reduce_each) sf = mod_symmetric(sf, em.mf, em.inv_m, em.lo, em.hi);
+            sum[BLK * 32 + i] = __float_as_uint(sf);
         }
     } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
             sum[BLK * 32 + i] += (uint32_t)ell * (uint32_t)__float2int_rn(__uint_as_float(v[i]) * em.acc_scale);
     }
+}
+
+// Write 32 rows x 128 bytes held one row per lane (chunk(c), c = 0..7, yields its 16-byte pieces) to global memory through a
+// 4 KB shared-memory block (16-byte chunks XOR-swizzled by row so neither pass has bank conflicts):
+// afterwards lane l holds chunk l%8 of rows l/8, l/8+4, ... and one store instruction covers 4 rows
+// x 128 contiguous bytes.  bytes_valid (<= 128, may be <= 0) is how much of the row piece lies
+// inside the matrix; pieces that are cut or rows that are not 16-byte aligned fall back to
+// element-wise stores.  With `add64` the 8-byte elements are added to what is already there.
+template <int elem, class ChunkFn>
+__device__ __forceinline__ void store_rows_128b(uint8_t* stage, int lane, ChunkFn chunk, uint8_t* gbase,
+                                                long long row_pitch, int rows_valid, int bytes_valid, int vec_ok,
+                                                bool add64) {
+    if (bytes_valid <= 0 || rows_valid <= 0) return;  // warp-uniform
+#pragma unroll
+    for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) = chunk(c);
+    __syncwarp();
+    const int c = lane & 7;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = i * 4 + (lane >> 3);
+        const uint4 v = *reinterpret_cast<const uint4*>(stage + r * 128 + ((c ^ (r & 7)) << 4));
+        if (r >= rows_valid) continue;
+        uint8_t* dst = gbase + r * row_pitch + c * 16;
+        if (vec_ok && c * 16 + 16 <= bytes_valid) {
+            if (add64) {
+                const longlong2 old = *reinterpret_cast<const longlong2*>(dst);
+                const long long a = (long long)(((unsigned long long)v.y << 32) | v.x) + old.x;
+                const long long b = (long long)(((unsigned long long)v.w << 32) | v.z) + old.y;
+                *reinterpret_cast<longlong2*>(dst) = make_longlong2(a, b);
+            } else {
+                *reinterpret_cast<uint4*>(dst) = v;
+            }
+        } else {
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 16 / elem; ++e) {
+                if (c * 16 + (e + 1) * elem > bytes_valid) continue;
+                if (elem == 4) {
+                    reinterpret_cast<uint32_t*>(dst)[e] = w[e];
+                } else if (elem == 2) {
+                    reinterpret_cast<uint16_t*>(dst)[e] = (uint16_t)(w[e >> 1] >> (16 * (e & 1)));
+                } else {
+                    const long long x = (long long)(((unsigned long long)w[2 * e + 1] << 32) | w[2 * e]);
+                    long long* d = reinterpret_cast<long long*>(dst) + e;
+                    *d = add64 ? *d + x : x;
+                }
+            }
+        }
+    }
+    __syncwarp();
 }
 
 template <bool kPair>
@@ -192,7 +265,8 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
-    Shared* sh = reinterpret_cast<Shared*>(smem_raw + (tiles_base - raw) + (size_t)kStages * kStageBytes);
+    Shared* sh = reinterpret_cast<Shared*>(smem_raw + (tiles_base - raw) + (size_t)kStages * kStageBytes +
+                                           (size_t)kEpiWarps * kStageWarpBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -335,9 +409,12 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int quarter = warp & 3, half = (warp - 2) >> 2;
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)half * 128u;
         const int m = p.modulus;
-        const float inv_m = m ? 1.0f / (float)m : 0.0f;
+        // symmetric representative of each coefficient keeps |l_k * residue| below m^2 / 4
+        const int m_hi = (m + 1) / 2 - 1;
         uint32_t drains = 0;
         bool ok = true;
+        // this warp's 4 KB staging block for the tile write-out
+        uint8_t* stage = smem_raw + (tiles_base - raw) + (size_t)kStages * kStageBytes + (size_t)(warp - 2) * kStageWarpBytes;
         // barriers the MMA issuer (CTA 0) waits on
         uint32_t acc_empty_bar[2], overlap_bar = ptx::smem_u32(&sh->overlap_free);
         for (int b = 0; b < 2; ++b) acc_empty_bar[b] = ptx::smem_u32(&sh->acc_empty[b]);
@@ -345,7 +422,18 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             overlap_bar = ptx::map_to_cta(overlap_bar, 0);
             for (int b = 0; b < 2; ++b) acc_empty_bar[b] = ptx::map_to_cta(acc_empty_bar[b], 0);
         }
-        const EpiMath em = {p.out_mode, m, inv_m, p.acc_scale};
+        EpiMath em = {};
+        em.out_mode = p.out_mode;
+        em.m = m;
+        em.acc_scale = p.acc_scale;
+        if (m) {
+            em.mf = (float)m;
+            em.inv_m = 1.0f / (float)m;
+            em.lo = (float)(-(m / 2));
+            em.hi = (float)m_hi;
+            // |sum| <= terms * (m/2)^2 must stay below 2^22
+            em.reduce_each = (long long)p.r * chunks * (m / 2 + 2) * (m / 2 + 2) >= (1ll << 22);
+        }
         for (int t = worker, tile_iter = 0; t < num_tiles && ok; t += num_workers, ++tile_iter) {
             int tm, tn;
             tile_coords(t, p.tiles_m, p.tiles_n, &tm, &tn);
@@ -353,7 +441,8 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
             for (int i = 0; i < 128; ++i) sum[i] = 0;
             for (int kk = 0; kk < p.r && ok; ++kk) {
-                const int ell = p.ell[product_at(kk, tile_iter, p.r)];
+                int ell = p.ell[product_at(kk, tile_iter, p.r)];
+                if (m && ell > m_hi) ell -= m;
                 for (int c = 0; c < chunks && ok; ++c, ++drains) {
                     const uint32_t ab = drains & 1u;
                     ok = bounded_wait(sh, ptx::smem_u32(&sh->acc_full[ab]), (drains >> 1) & 1u, p.status, 4);
@@ -364,14 +453,12 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     // (held by the warps of column half 1) and the first block of accumulator 1 (half 0):
                     // they are read first and handed back at once.
                     if (ab == 0) {
-                        drain_block<3>(taddr + kAccCol0, sum, em, ell);
-                        if (half == 1) release(overlap_bar, lane, kPair);
+                        drain_block<3>(taddr + kAccCol0, sum, em, ell, half == 1 ? overlap_bar : 0u, lane, kPair);
                         drain_block<0>(taddr + kAccCol0, sum, em, ell);
                         drain_block<1>(taddr + kAccCol0, sum, em, ell);
                         drain_block<2>(taddr + kAccCol0, sum, em, ell);
                     } else {
-                        drain_block<0>(taddr + kAccCol1, sum, em, ell);
-                        if (half == 0) release(overlap_bar, lane, kPair);
+                        drain_block<0>(taddr + kAccCol1, sum, em, ell, half == 0 ? overlap_bar : 0u, lane, kPair);
                         drain_block<1>(taddr + kAccCol1, sum, em, ell);
                         drain_block<2>(taddr + kAccCol1, sum, em, ell);
                         drain_block<3>(taddr + kAccCol1, sum, em, ell);
@@ -380,70 +467,61 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 }
             }
             if (!ok) break;
-            // ---- write the tile: this thread owns one row and 128 consecutive columns
-            const long long row = (long long)(tm * C::kCtas + (int)rank) * kTileM + quarter * 32 + lane;
+            // ---- write the tile.  This thread owns one row and 128 consecutive columns; the warp
+            // passes every 128-byte row piece through its shared-memory staging block so that each store
+            // instruction writes 4 rows x 128 contiguous bytes instead of 32 rows x 16 bytes.
+            const long long row0 = (long long)(tm * C::kCtas + (int)rank) * kTileM + quarter * 32;  // first row of the warp
             const int col0 = tn * kTileN + half * 128;
-            if (row < p.M) {
-                const int ncols = min(128, p.N - col0);
-                const int hi_res = (m + 1) / 2 - 1;
-                if (p.out_mode == OUT_I32 || p.out_mode == OUT_RES_I32 || p.out_mode == OUT_RAW_F32) {
-                    uint32_t* dst = reinterpret_cast<uint32_t*>(p.C) + row * p.ldc + col0;
+            const int rows_valid = (int)max(0ll, min(32ll, (long long)p.M - row0));
+            if (m) {
+                // residue sums are floats: one last reduction, then to integers in the symmetric range
 #pragma unroll
-                    for (int i = 0; i < 128; i += 4) {
+                for (int i = 0; i < 128; ++i)
+                    sum[i] = __float_as_uint(mod_symmetric(__uint_as_float(sum[i]), em.mf, em.inv_m, em.lo, em.hi) +
+                                             12582912.0f) - 0x4B400000u;  // float -> int
+            }
+            if (p.out_mode == OUT_I32 || p.out_mode == OUT_RES_I32 || p.out_mode == OUT_RAW_F32) {
+                uint8_t* gbase = reinterpret_cast<uint8_t*>(p.C) + (row0 * p.ldc + col0) * 4;
+#pragma unroll
+                for (int blk = 0; blk < 4; ++blk) {  // 32 columns = 128 bytes per row
+                    const bool shift = p.out_mode == OUT_I32;
+                    auto chunk = [&](int c) {
                         uint32_t o[4];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            uint32_t x = sum[i + j];
-                            if (p.out_mode == OUT_I32) x = (uint32_t)((int)x >> p.log2D);
-                            if (p.out_mode == OUT_RES_I32) x = (uint32_t)((int)x > hi_res ? (int)x - m : (int)x);
-                            o[j] = x;
+                            const uint32_t x = sum[blk * 32 + c * 4 + j];
+                            o[j] = shift ? (uint32_t)((int)x >> p.log2D) : x;
                         }
-                        if (p.vec_store && i + 4 <= ncols) {
-                            *reinterpret_cast<uint4*>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
-                        } else {
+                        return make_uint4(o[0], o[1], o[2], o[3]);
+                    };
+                    store_rows_128b<4>(stage, lane, chunk, gbase + blk * 128, p.ldc * 4, rows_valid,
+                                       (p.N - col0 - blk * 32) * 4, p.vec_store, false);
+                }
+            } else if (p.out_mode == OUT_I64) {
+                uint8_t* gbase = reinterpret_cast<uint8_t*>(p.C) + (row0 * p.ldc + col0) * 8;
 #pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                if (i + j < ncols) dst[i + j] = o[j];
-                        }
-                    }
-                } else if (p.out_mode == OUT_I64) {
-                    long long* dst = reinterpret_cast<long long*>(p.C) + row * p.ldc + col0;
+                for (int blk = 0; blk < 8; ++blk) {  // 16 columns = 128 bytes per row
+                    auto chunk = [&](int c) {
+                        const long long o0 = (long long)((int)sum[blk * 16 + c * 2] >> p.log2D);
+                        const long long o1 = (long long)((int)sum[blk * 16 + c * 2 + 1] >> p.log2D);
+                        return make_uint4((uint32_t)o0, (uint32_t)(o0 >> 32), (uint32_t)o1, (uint32_t)(o1 >> 32));
+                    };
+                    store_rows_128b<8>(stage, lane, chunk, gbase + blk * 128, p.ldc * 8, rows_valid,
+                                       (p.N - col0 - blk * 16) * 8, p.vec_store, p.accumulate != 0);
+                }
+            } else {  // OUT_RES_I16
+                uint8_t* gbase = reinterpret_cast<uint8_t*>(p.C) + (row0 * p.ldc + col0) * 2;
 #pragma unroll
-                    for (int i = 0; i < 128; i += 2) {
-                        long long o0 = (long long)((int)sum[i] >> p.log2D);
-                        long long o1 = (long long)((int)sum[i + 1] >> p.log2D);
-                        if (p.vec_store && i + 2 <= ncols) {
-                            if (p.accumulate) {
-                                const longlong2 old = *reinterpret_cast<longlong2*>(dst + i);
-                                o0 += old.x;
-                                o1 += old.y;
-                            }
-                            *reinterpret_cast<longlong2*>(dst + i) = make_longlong2(o0, o1);
-                        } else {
-                            if (i < ncols) dst[i] = p.accumulate ? dst[i] + o0 : o0;
-                            if (i + 1 < ncols) dst[i + 1] = p.accumulate ? dst[i + 1] + o1 : o1;
-                        }
-                    }
-                } else {  // OUT_RES_I16
-                    short* dst = reinterpret_cast<short*>(p.C) + row * p.ldc + col0;
-#pragma unroll
-                    for (int i = 0; i < 128; i += 8) {
+                for (int blk = 0; blk < 2; ++blk) {  // 64 columns = 128 bytes per row
+                    auto chunk = [&](int c) {
                         uint32_t w[4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            int x0 = (int)sum[i + 2 * j], x1 = (int)sum[i + 2 * j + 1];
-                            x0 = x0 > hi_res ? x0 - m : x0;
-                            x1 = x1 > hi_res ? x1 - m : x1;
-                            w[j] = ((uint32_t)x0 & 0xFFFFu) | ((uint32_t)x1 << 16);
-                        }
-                        if (p.vec_store && i + 8 <= ncols) {
-                            *reinterpret_cast<uint4*>(dst + i) = make_uint4(w[0], w[1], w[2], w[3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                if (i + j < ncols) dst[i + j] = (short)((w[j >> 1] >> (16 * (j & 1))) & 0xFFFFu);
-                        }
-                    }
+                        for (int j = 0; j < 4; ++j)
+                            w[j] = (sum[blk * 64 + c * 8 + 2 * j] & 0xFFFFu) | (sum[blk * 64 + c * 8 + 2 * j + 1] << 16);
+                        return make_uint4(w[0], w[1], w[2], w[3]);
+                    };
+                    store_rows_128b<2>(stage, lane, chunk, gbase + blk * 128, p.ldc * 2, rows_valid,
+                                       (p.N - col0 - blk * 64) * 2, p.vec_store, false);
                 }
             }
         }
@@ -524,7 +602,11 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair>, ma, mb, p) != cudaSuccess) return AWE_ERR_CUDA;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair>, ma, mb, p);
+    if (err != cudaSuccess) {
+        if (getenv("AWE_DEBUG")) fprintf(stderr, "awe: GEMM launch failed: %s\n", cudaGetErrorString(err));
+        return AWE_ERR_CUDA;
+    }
     h->launches += 1;
     return AWE_OK;
 }
@@ -589,6 +671,8 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
     p.sf_word = kScaleWord;
     // exact accumulation segment (Section 3.4): a multiple of 256 not above K*
     int64_t kc = k_chunk ? k_chunk : std::max<int64_t>(256, d.k_star / 256 * 256);
+    // the residue epilogue works on partial sums below 2^22 (see mod_symmetric)
+    if (residue) kc = std::min<int64_t>(kc, std::max<int64_t>(256, d.k_star / 4 / 256 * 256));
     p.chunk_kblocks = (int)std::min<int64_t>(kc / 256, 1 << 20);
     const int64_t total_kblocks = pitch / kBlockKBytes;
     // 64-bit results: K is cut into launches whose own result fits 32 bits, added in int64

@@ -85,6 +85,24 @@ Scheme make_awe4() {
     return s;
 }
 
+Scheme make_ternary() {
+    // A in {-1,0,1} is a single limb; B = b0 + 13 b1 + 169 b2; AB = P0 + 13 P1 + 169 P2 (Section 6.2)
+    Scheme s;
+    s.p = 1;
+    s.q = 3;
+    s.r = 3;
+    s.w[0] = 1;
+    set_vec(s.v, {1, 13, 169});
+    for (int k = 0; k < 3; ++k) {
+        s.alpha[k][0] = 1;
+        s.beta[k][k] = 1;
+    }
+    set_vec(s.ell, {1, 13, 169});
+    s.a_lo = -1;
+    s.a_hi = 1;
+    return s;
+}
+
 struct Choice {
     int max_abs, sum_abs;
     int limbs[kMaxLimbs];
@@ -242,7 +260,9 @@ std::map<std::tuple<int, int, int, int>, SideTable> g_tables;
 }  // namespace
 
 awe_in_dtype_t natural_dtype(int enc, awe_side_t side) {
-    return (enc == AWE_ENC_INT4xINT8_AWE4 && side == AWE_SIDE_A) ? AWE_I4_IN_I8 : AWE_I8;
+    if (enc == AWE_ENC_INT4xINT8_AWE4 && side == AWE_SIDE_A) return AWE_I4_IN_I8;
+    if (enc == AWE_ENC_TERNARY_INT8_3 && side == AWE_SIDE_A) return AWE_T2_IN_I8;
+    return AWE_I8;
 }
 
 bool get_scheme(int enc, int modulus, Scheme* out) {
@@ -271,6 +291,10 @@ bool get_scheme(int enc, int modulus, Scheme* out) {
             break;
         case AWE_ENC_INT4xINT8_AWE4:
             s = make_awe4();
+            ok = true;
+            break;
+        case AWE_ENC_TERNARY_INT8_3:
+            s = make_ternary();
             ok = true;
             break;
         case AWE_ENC_MOD_M:
@@ -309,6 +333,7 @@ bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, co
     for (int b = 0; b < 256; ++b) {
         int x = (int)(int8_t)b;
         if (dt == AWE_I4_IN_I8) x = (int)(int8_t)((b & 0xF) << 4) >> 4;  // low nibble, sign-extended
+        if (dt == AWE_T2_IN_I8 && (x < -1 || x > 1)) x = 0;              // not a ternary value
         int key_x = x;
         if (s.modulus) {
             key_x = ((x % s.modulus) + s.modulus) % s.modulus;
@@ -367,7 +392,7 @@ extern "C" awe_status_t awe_encoding_info(int enc, int modulus, awe_encoding_des
 
 extern "C" awe_status_t awe_encoding_lut(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt,
                                          int8_t* lut_host) {
-    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (dt != AWE_I8 && dt != AWE_I4_IN_I8))
+    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (int)dt < 0 || (int)dt > 2)
         return AWE_ERR_INVALID_ARG;
     const SideTable* t;
     if (!get_side_table(enc, modulus, side, dt, &t)) return AWE_ERR_UNSUPPORTED;

@@ -100,6 +100,23 @@ def test_int4_x_int8():
         assert np.array_equal(got, mm.matmul_i64(A, B))
 
 
+def test_ternary_x_int8():
+    """Section 6.2: {0, +-1} x INT8 in 3 products (one limb against the three base-13 limbs)."""
+    for (M, N, K) in [(256, 512, 1024), (130, 270, 300), (1, 1, 1)]:
+        A, B = wl.make_inputs(wl.small("t", M, N, K, "ternary", "int8", seed=19))
+        got = gu.gpu_gemm_exact(A, B, b.ENC_TERNARY_INT8_3, b.C_I32, a_dt=b.T2_IN_I8)
+        assert np.array_equal(got, mm.matmul_i64(A, B))
+        assert np.array_equal(got, pl.awe_matmul(sc.TERNARY3, A, B, a_range=(-1, 1)))
+    # bytes that are not ternary values are read as 0
+    A, B = wl.make_inputs(wl.small("t", 128, 256, 256, "ternary", "int8", seed=20))
+    dirty = A.copy()
+    dirty[::3, ::5] = 77
+    clean = dirty.copy()
+    clean[clean == 77] = 0
+    assert np.array_equal(gu.gpu_gemm_exact(dirty, B, b.ENC_TERNARY_INT8_3, b.C_I32, a_dt=b.T2_IN_I8),
+                          mm.matmul_i64(clean, B))
+
+
 @pytest.mark.parametrize("m", rns.RNS_SET_FP64)
 def test_residue_form_every_modulus_of_the_set(m):
     A, B = wl.make_inputs(wl.small("t", 192, 320, 1100, "residue", "residue", seed=m, modulus=m))

@@ -37,6 +37,10 @@ def test_records_match_the_paper_and_the_oracle(b):
         assert d.r == s.r and list(d.ell)[:d.r] == list(s.ell) and d.log2D == s.log2D
         assert list(d.ia)[:d.r] == s.plane_index("A") and list(d.ib)[:d.r] == s.plane_index("B")
         assert d.n_planes_a == len(s.stored_planes("A")) and d.n_planes_b == len(s.stored_planes("B"))
+    d = b.awe_encoding_info(b.ENC_TERNARY_INT8_3)
+    s = sc.TERNARY3
+    assert d.r == 3 and list(d.ell)[:3] == list(s.ell) and list(d.ib)[:3] == s.plane_index("B")
+    assert (d.n_planes_a, d.n_planes_b, d.c_a, d.c_b, d.k_star) == (1, 3, 1, 8, 2097152)
     d = b.awe_encoding_info(b.ENC_INT8_AWE6)
     assert (d.c_a, d.c_b, d.k_star) == (6, 6, 466033)
     d = b.awe_encoding_info(b.ENC_INT4xINT8_AWE4)
@@ -52,6 +56,11 @@ def test_tables_match_the_oracle_tables(b):
     assert np.array_equal(lut[np.arange(-8, 8) & 0xFF], pl.plane_lut(sc.AWE4, "A", -8, 7))
     assert np.array_equal(b.awe_encoding_lut(b.ENC_INT4xINT8_AWE4, 0, b.SIDE_B)[idx],
                           pl.plane_lut(sc.AWE4, "B", -128, 127))
+    lut = b.awe_encoding_lut(b.ENC_TERNARY_INT8_3, 0, b.SIDE_A, b.T2_IN_I8)
+    assert np.array_equal(lut[np.arange(-1, 2) & 0xFF], pl.plane_lut(sc.TERNARY3, "A", -1, 1))
+    assert not lut[2:255].any()                                   # non-ternary bytes are read as 0
+    assert np.array_equal(b.awe_encoding_lut(b.ENC_TERNARY_INT8_3, 0, b.SIDE_B)[idx],
+                          pl.plane_lut(sc.TERNARY3, "B", -128, 127))
     for m in rns.RNS_SET_FP64 + (2, 10, 37, 91, 100, 169):
         s = sc.mod_scheme(m)
         d = b.awe_encoding_info(b.ENC_MOD_M, m)
