@@ -14,7 +14,7 @@ configuration uses.
 from __future__ import annotations
 
 import math
-from typing import Dict, List, Tuple
+from typing import Dict, List, Sequence, Tuple
 
 import numpy as np
 
@@ -62,3 +62,51 @@ def select_moduli(costs: Dict[int, int], width: int = 54, K: int = 16384) -> Tup
 # The set the residue configuration runs (width 54, K = 16,384): 5 one-product, 13
 # three-product and 4 four-product moduli, 60 products.
 RNS_SET_FP64 = (7, 8, 9, 11, 13, 41, 43, 47, 53, 59, 61, 67, 71, 73, 79, 83, 85, 89, 139, 149, 151, 157)
+
+
+# --------------------------------------------------------------------------- wide integers
+# Section 5.3: a residue number system splits the inputs into residues modulo pairwise coprime
+# moduli, computes the per-modulus products in parallel and reconstructs by the Chinese remainder
+# theorem; unique reconstruction of the accumulated product requires prod(m) > 2 K B_A B_B.
+def residues(X, m: int) -> np.ndarray:
+    """Entrywise symmetric residue of an integer array (any integer dtype or Python ints), int8."""
+    lo = -(m // 2)
+    flat = [((int(x) - lo) % m) + lo for x in np.asarray(X, dtype=object).ravel()]
+    return np.array(flat, dtype=np.int8).reshape(np.shape(X))
+
+
+def crt_symmetric(res: Sequence[int], moduli: Sequence[int]) -> int:
+    """The integer x with |x| <= prod(m)/2 and x = res[t] (mod moduli[t]) for every t, by the
+    textbook formula x = sum_t res_t M_t (M_t^-1 mod m_t) mod M with M_t = M / m_t."""
+    M = math.prod(moduli)
+    x = 0
+    for r, m in zip(res, moduli):
+        Mt = M // m
+        x += int(r) * Mt * pow(Mt, -1, m)
+    x %= M
+    return x - M if x > M // 2 else x
+
+
+def wide_matmul(A, B) -> np.ndarray:
+    """The definition: exact product of integer matrices in unbounded Python integers."""
+    return np.asarray(A, dtype=object) @ np.asarray(B, dtype=object)
+
+
+def rns_matmul(A, B, moduli: Sequence[int] = RNS_SET_FP64, width: int = 54) -> np.ndarray:
+    """The method of Section 5.3 step by step: residues, one residue product per modulus through
+    Algorithm 1 (mod-m scheme), CRT.  A: M x K, B: K x N integers of the given width."""
+    from . import pipeline
+    A = np.asarray(A, dtype=object)
+    B = np.asarray(B, dtype=object)
+    K = A.shape[1]
+    bound = 2 ** (width - 1) - 1
+    assert all(abs(int(x)) <= bound for x in A.ravel()) and all(abs(int(x)) <= bound for x in B.ravel())
+    assert math.prod(moduli) > 2 * K * bound * bound, "moduli too small for a unique result"
+    per_mod = []
+    for m in moduli:
+        s = mod_scheme(m)
+        per_mod.append(pipeline.awe_matmul(s, residues(A, m), residues(B, m)))
+    out = np.empty(per_mod[0].shape, dtype=object)
+    for idx in np.ndindex(*out.shape):
+        out[idx] = crt_symmetric([int(c[idx]) for c in per_mod], moduli)
+    return out

@@ -97,3 +97,43 @@ def test_integer_program_reaches_the_same_total():
     total, sel = rns.select_moduli(costs)
     assert total == 60
     assert sum(costs[m] for m in sel) == total
+
+
+# ------------------------------------------------------------------ residue number system, wide integers
+def test_crt_textbook_examples():
+    # Sunzi's problem: x = 2 (mod 3), 3 (mod 5), 2 (mod 7) -> 23
+    assert rns.crt_symmetric([2, 3, 2], [3, 5, 7]) == 23
+    assert rns.crt_symmetric([-1, -1, -1], [3, 5, 7]) == -1
+    assert rns.crt_symmetric([1, 2, 3, 4], [5, 7, 9, 11]) % 5 == 1
+    M = math.prod(rns.RNS_SET_FP64)
+    rng = np.random.default_rng(9)
+    for _ in range(50):
+        x = int(rng.integers(-2 ** 62, 2 ** 62)) * int(rng.integers(1, 2 ** 58)) + int(rng.integers(0, 2 ** 40))
+        assert abs(x) < M // 2
+        res = [int(rns.residues(np.array([x], dtype=object), m)[0]) for m in rns.RNS_SET_FP64]
+        assert rns.crt_symmetric(res, rns.RNS_SET_FP64) == x
+
+
+def test_residues_are_symmetric_and_congruent():
+    xs = np.array([-(2 ** 53 - 1), -12345678901234, -1, 0, 1, 77, 2 ** 53 - 1], dtype=np.int64)
+    for m in (7, 8, 157):
+        r = rns.residues(xs, m)
+        lo, hi = sc.symmetric_range(m)
+        assert r.min() >= lo and r.max() <= hi
+        assert all((int(x) - int(y)) % m == 0 for x, y in zip(xs, r))
+
+
+def test_rns_product_of_width_54_integers_equals_the_definition():
+    rng = np.random.default_rng(10)
+    B53 = 2 ** 53 - 1
+    A = rng.integers(-B53, B53 + 1, (5, 9), dtype=np.int64)
+    B = rng.integers(-B53, B53 + 1, (9, 4), dtype=np.int64)
+    A[0, :] = B53                                       # largest magnitudes, all signs aligned
+    B[:, 0] = -B53
+    want = rns.wide_matmul(A, B)
+    assert want[0, 0] == -9 * B53 * B53
+    got = rns.rns_matmul(A, B)
+    assert all(int(got[i]) == int(want[i]) for i in np.ndindex(*want.shape))
+    # a modulus set that is too small must be refused (uniqueness condition of Section 5.3)
+    with pytest.raises(AssertionError):
+        rns.rns_matmul(A, B, moduli=rns.RNS_SET_FP64[:-4])
