@@ -381,6 +381,41 @@ def main():
                 del am, bm
             ctx["residue_22_moduli_8192_total_ms"] = total_ms
             ctx["residue_22_moduli_fp4_gemms"] = prods
+            # width-54 integers (the FP64 significand) through the residue number system + CRT
+            B53 = 2 ** 53 - 1
+            aw = torch.randint(-B53, B53 + 1, (8192, 8192), dtype=torch.int64, device=dev, generator=gen)
+            bw = torch.randint(-B53, B53 + 1, (8192, 8192), dtype=torch.int64, device=dev, generator=gen)
+            wsw = torch.empty(b.awe_wide_workspace_bytes(8192, 8192, 8192), dtype=torch.uint8, device=dev)
+            cw = torch.empty((8192, 8192, 2), dtype=torch.int64, device=dev)
+            nmod = len(RNS_SET_FP64)
+            ra = torch.empty((nmod, 8192 * 8192), dtype=torch.int8, device=dev)
+            rc = torch.empty((nmod, 8192 * 8192), dtype=torch.int16, device=dev)
+            for _ in range(2):
+                b.awe_gemm_exact_wide(h, aw, bw, 8192, 8192, 8192, 54, cw, wsw)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(3):
+                b.awe_gemm_exact_wide(h, aw, bw, 8192, 8192, 8192, 54, cw, wsw)
+            e1.record()
+            torch.cuda.synchronize()
+            ms_wide = e0.elapsed_time(e1) / 3
+            e0.record()
+            for _ in range(3):
+                b.awe_wide_residues(h, aw, 8192 * 8192, ra)
+            e1.record()
+            torch.cuda.synchronize()
+            ms_res = e0.elapsed_time(e1) / 3
+            e0.record()
+            for _ in range(3):
+                b.awe_wide_crt(h, rc, 8192 * 8192, cw)
+            e1.record()
+            torch.cuda.synchronize()
+            ms_crt = e0.elapsed_time(e1) / 3
+            ctx["wide_int54_8192"] = {"total_ms": ms_wide, "effective_TOPS": ops / (ms_wide * 1e-3) / 1e12,
+                                      "residues_one_operand_ms": ms_res, "crt_ms": ms_crt,
+                                      "residues_GBs": 8192 * 8192 * (8 + nmod) / (ms_res * 1e-3) / 1e9,
+                                      "crt_GBs": 8192 * 8192 * (2 * nmod + 16) / (ms_crt * 1e-3) / 1e9}
+            del aw, bw, wsw, cw, ra, rc
         ctx["paper_theoretical_TOPS"] = "1500 (9.0 PFLOPS / 6, published peak, not a measurement; B200)"
         line["context"] = ctx
 

@@ -163,6 +163,39 @@ awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, awe_in_dtyp
                                  void* C_host, awe_out_dtype_t out_dt, void* scratch_dev, size_t scratch_bytes,
                                  void* stream);
 
+/* ---- Wide integers through a residue number system (Section 5.3; Table I, "FP64 significand").
+ * The inputs are split into symmetric residues modulo pairwise coprime moduli, each residue product
+ * runs as a mod-m product on the FP4 kernels, and the Chinese remainder theorem rebuilds the exact
+ * integers.  The built-in set has 22 moduli (60 FP4 GEMMs) with product 2^122.86, which gives a
+ * unique result whenever 2 K (2^(in_bits-1) - 1)^2 stays below it: in_bits = 54 up to K = 59,000. */
+
+/* The moduli of the built-in set: writes up to `capacity` of them to out (may be NULL), returns
+ * how many there are.  Host only. */
+int awe_wide_moduli(int32_t* out, int capacity);
+
+/* Bytes of scratch awe_gemm_exact_wide needs: residues of A and B (int8, one copy per modulus),
+ * the residue products (int16 per modulus) and the plane workspace of one modulus. */
+size_t awe_wide_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
+/* Symmetric residues of `count` 64-bit integers (|x| < 2^56) for every modulus of the set:
+ * res_dev[t * count + i] = X_dev[i] mod m_t in [-floor(m_t/2), ceil(m_t/2) - 1], int8.  Elementwise, so
+ * the residue arrays keep the layout of X.  X_dev 16-B aligned, res_dev 4-B aligned. */
+awe_status_t awe_wide_residues(awe_handle_t h, const int64_t* X_dev, int64_t count, int8_t* res_dev, void* stream);
+
+/* Chinese-remainder reconstruction: res_dev[t * count + i] (int16) is the symmetric residue of the
+ * unknown integer x_i modulo m_t; writes x_i, the representative with |x_i| <= prod(m)/2, as a
+ * 128-bit two's-complement integer: out_dev[2 i] = low 64 bits, out_dev[2 i + 1] = high 64 bits. */
+awe_status_t awe_wide_crt(awe_handle_t h, const int16_t* res_dev, int64_t count, int64_t* out_dev, void* stream);
+
+/* C = A.B exactly for integer matrices whose entries satisfy |x| <= 2^(in_bits-1) - 1, in_bits <= 54.
+ * A_dev: M x K int64 row-major, B_dev: K x N int64 row-major, C_dev: M x N 128-bit integers (two
+ * int64 each, low word first).  AWE_ERR_RANGE if the moduli cannot hold the result for this K.
+ * workspace_dev: awe_wide_workspace_bytes bytes, 256-B aligned.  Inputs outside the stated width
+ * give an unspecified result (they are not checked on the device). */
+awe_status_t awe_gemm_exact_wide(awe_handle_t h, const int64_t* A_dev, const int64_t* B_dev, int64_t M, int64_t N,
+                                 int64_t K, int in_bits, int64_t* C_dev, void* workspace_dev, size_t workspace_bytes,
+                                 void* stream);
+
 /* Largest awe_workspace_bytes() a problem may need to go through awe_gemm_exact_static: 24 MiB,
  * e.g. INT8xINT8 with the 6-product encoding up to M = N = K = 2048. */
 #define AWE_STATIC_WORKSPACE_BYTES (24u << 20)

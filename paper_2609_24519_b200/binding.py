@@ -29,7 +29,8 @@ STATIC_WORKSPACE_BYTES = 24 << 20
 
 EXPORTS = ["awe_create", "awe_destroy", "awe_encoding_info", "awe_encoding_lut", "awe_planes_bytes",
            "awe_workspace_bytes", "awe_host_staging_bytes", "awe_encode", "awe_gemm_planes", "awe_gemm_exact",
-           "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_fp4_product_raw", "awe_last_device_status", "awe_last_gemm_clock_mhz", "awe_launch_count",
+           "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_wide_moduli", "awe_wide_workspace_bytes",
+           "awe_wide_residues", "awe_wide_crt", "awe_gemm_exact_wide", "awe_fp4_product_raw", "awe_last_device_status", "awe_last_gemm_clock_mhz", "awe_launch_count",
            "awe_status_string"]
 
 
@@ -75,6 +76,12 @@ def lib() -> ctypes.CDLL:
     L.awe_gemm_exact.argtypes = [vp, vp, i32, vp, i32, i64, i64, i64, i32, i32, vp, i32, vp, sz, vp]
     L.awe_gemm_exact_host.argtypes = [vp, vp, i32, vp, i32, i64, i64, i64, i32, i32, vp, i32, vp, sz, vp]
     L.awe_gemm_exact_static.argtypes = [vp, i32, vp, i32, i64, i64, i64, i32, i32, vp, i32, vp]
+    L.awe_wide_moduli.argtypes = [vp, i32]
+    L.awe_wide_workspace_bytes.argtypes = [i64, i64, i64]
+    L.awe_wide_workspace_bytes.restype = sz
+    L.awe_wide_residues.argtypes = [vp, vp, i64, vp, vp]
+    L.awe_wide_crt.argtypes = [vp, vp, i64, vp, vp]
+    L.awe_gemm_exact_wide.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, sz, vp]
     L.awe_fp4_product_raw.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
     L.awe_last_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.awe_last_gemm_clock_mhz.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
@@ -210,6 +217,33 @@ def awe_gemm_exact_static(A, a_dt: int, B, b_dt: int, M: int, N: int, K: int, en
     Runs on the current CUDA device; calls that could overlap on the GPU must be serialised."""
     _check(lib().awe_gemm_exact_static(_ptr(A), a_dt, _ptr(B), b_dt, M, N, K, enc, modulus, _ptr(C), out_dt,
                                        _stream(stream)), "awe_gemm_exact_static")
+
+
+def awe_wide_moduli():
+    n = lib().awe_wide_moduli(None, 0)
+    out = (ctypes.c_int32 * n)()
+    lib().awe_wide_moduli(out, n)
+    return list(out)
+
+
+def awe_wide_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib().awe_wide_workspace_bytes(M, N, K))
+
+
+def awe_wide_residues(h: Handle, X, count: int, res, stream=None) -> None:
+    _check(lib().awe_wide_residues(h.raw, _ptr(X), count, _ptr(res), _stream(stream)), "awe_wide_residues")
+
+
+def awe_wide_crt(h: Handle, res, count: int, out, stream=None) -> None:
+    _check(lib().awe_wide_crt(h.raw, _ptr(res), count, _ptr(out), _stream(stream)), "awe_wide_crt")
+
+
+def awe_gemm_exact_wide(h: Handle, A, B, M: int, N: int, K: int, in_bits: int, C, workspace,
+                        workspace_bytes: Optional[int] = None, stream=None) -> None:
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().awe_gemm_exact_wide(h.raw, _ptr(A), _ptr(B), M, N, K, in_bits, _ptr(C), _ptr(workspace),
+                                     workspace_bytes, _stream(stream)), "awe_gemm_exact_wide")
 
 
 def awe_fp4_product_raw(h: Handle, planeX, planeY, M: int, N: int, K: int, P, ldp: int, stream=None) -> None:

@@ -1,0 +1,280 @@
+// Exact product of wide-integer matrices through a residue number system (Section 5.3):
+// residues of both operands modulo pairwise coprime moduli, one residue product per modulus on the
+// FP4 kernels (mod-m schemes), reconstruction by the Chinese remainder theorem.  For input width 54
+// (the FP64 significand) the built-in set has 22 moduli and needs 60 FP4 GEMMs.
+#include <cmath>
+#include <cstring>
+
+#include "awe_internal.h"
+
+using namespace awe;
+
+namespace {
+
+constexpr int kMaxModuli = 32;
+// 5 one-product, 13 three-product and 4 four-product moduli; product = 2^122.86.
+const int kWideModuli[] = {7, 8, 9, 11, 13, 41, 43, 47, 53, 59, 61, 67, 71, 73, 79, 83, 85, 89, 139, 149, 151, 157};
+constexpr int kNumWideModuli = sizeof(kWideModuli) / sizeof(int);
+
+typedef unsigned __int128 u128;
+typedef __int128 i128;
+
+struct ResidueParams {
+    int n;
+    int m[kMaxModuli];
+    unsigned int c1[kMaxModuli], c2[kMaxModuli], c3[kMaxModuli];  // 2^14, 2^28, 2^42 mod m
+    unsigned int magic[kMaxModuli];                                // floor((2^32 - 1) / m) + 1
+};
+
+// |x| < 2^56 as four 14-bit limbs l0..l3: |x| = l0 + l1 2^14 + l2 2^28 + l3 2^42.
+struct Limbs14 {
+    unsigned int l0, l1, l2, l3;
+    bool neg;
+};
+
+__device__ __forceinline__ Limbs14 split14(long long x) {
+    const unsigned long long ax = x < 0 ? (unsigned long long)(-x) : (unsigned long long)x;
+    Limbs14 r;
+    r.l0 = (unsigned int)ax & 0x3FFFu;
+    r.l1 = (unsigned int)(ax >> 14) & 0x3FFFu;
+    r.l2 = (unsigned int)(ax >> 28) & 0x3FFFu;
+    r.l3 = (unsigned int)(ax >> 42) & 0x3FFFu;
+    r.neg = x < 0;
+    return r;
+}
+
+// x mod m in the symmetric range.  s = l0 + l1 c1 + l2 c2 + l3 c3 is congruent to |x| and stays
+// below 2^23, where the 32-bit multiply-high by ceil(2^32 / m) gives the exact quotient.
+__device__ __forceinline__ int symmetric_residue(const Limbs14& v, int m, unsigned int c1, unsigned int c2,
+                                                 unsigned int c3, unsigned int magic) {
+    const unsigned int s = v.l0 + v.l1 * c1 + v.l2 * c2 + v.l3 * c3;
+    int r = (int)(s - __umulhi(s, magic) * (unsigned int)m);  // in [0, m)
+    if (v.neg && r != 0) r = m - r;
+    return r > (m + 1) / 2 - 1 ? r - m : r;
+}
+
+// X: `count` 64-bit integers; out[t * count + i] = symmetric residue of X[i] modulo m[t].
+// A thread takes 4 consecutive elements so every store is a 4-byte word and a warp writes 128
+// contiguous bytes per modulus.
+__global__ void __launch_bounds__(256)
+wide_residues_kernel(const long long* __restrict__ X, long long count, const __grid_constant__ ResidueParams p,
+                     int8_t* __restrict__ out) {
+    const long long groups = (count + 3) / 4;
+    for (long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
+         g += (long long)gridDim.x * blockDim.x) {
+        const long long i0 = g * 4;
+        long long x[4] = {0, 0, 0, 0};
+        if (i0 + 4 <= count) {
+            const longlong2 a = __ldg(reinterpret_cast<const longlong2*>(X + i0));
+            const longlong2 b = __ldg(reinterpret_cast<const longlong2*>(X + i0) + 1);
+            x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
+        } else {
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j < count) x[j] = X[i0 + j];
+        }
+        Limbs14 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = split14(x[j]);
+        const bool full = (i0 + 4 <= count) && ((count & 3) == 0);
+        for (int t = 0; t < p.n; ++t) {
+            const int m = p.m[t];
+            uint32_t word = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                word |= ((uint32_t)symmetric_residue(v[j], m, p.c1[t], p.c2[t], p.c3[t], p.magic[t]) & 0xFFu) << (8 * j);
+            int8_t* dst = out + (long long)t * count + i0;
+            if (full) {
+                *reinterpret_cast<uint32_t*>(dst) = word;
+            } else {
+                for (int j = 0; j < 4; ++j)
+                    if (i0 + j < count) dst[j] = (int8_t)(word >> (8 * j));
+            }
+        }
+    }
+}
+
+struct CrtParams {
+    int n;
+    int m[kMaxModuli];
+    unsigned int w[kMaxModuli][4];  // W_t = (M/m_t) ((M/m_t)^-1 mod m_t) < 2^123 in four 32-bit limbs
+    unsigned int M[4];              // M = prod m_t
+    unsigned long long M_lo, M_hi, half_lo, half_hi;
+    double M_as_double;
+};
+
+// res[t * count + i]: symmetric residues of the unknown integers modulo m_t.  The integer with
+// -M/2 < x <= M/2 is x = sum_t r_t W_t mod M (textbook CRT) with r_t taken in [0, m_t).  The sum is
+// formed limb by limb (four 64-bit accumulators of 32 x 32-bit products, no carries needed: 22 terms
+// below 2^40 each), the quotient by M (< 2^13) is estimated in double precision, q M is subtracted
+// limb by limb, carries are propagated once, and at most two corrections fix the estimate.
+__global__ void __launch_bounds__(256)
+wide_crt_kernel(const short* __restrict__ res, long long count, const __grid_constant__ CrtParams p,
+                long long* __restrict__ out) {
+    const i128 M = (i128)(((u128)p.M_hi << 64) | p.M_lo);
+    const i128 half = (i128)(((u128)p.half_hi << 64) | p.half_lo);
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count;
+         i += (long long)gridDim.x * blockDim.x) {
+        unsigned long long a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+#pragma unroll 2
+        for (int t = 0; t < p.n; ++t) {
+            int r = (int)res[(long long)t * count + i];
+            r += r < 0 ? p.m[t] : 0;
+            const unsigned int ru = (unsigned int)r;
+            a0 += (unsigned long long)ru * p.w[t][0];
+            a1 += (unsigned long long)ru * p.w[t][1];
+            a2 += (unsigned long long)ru * p.w[t][2];
+            a3 += (unsigned long long)ru * p.w[t][3];
+        }
+        const double xd = ((double)a3 * 4294967296.0 + (double)a2) * 18446744073709551616.0 +
+                          (double)a1 * 4294967296.0 + (double)a0;
+        const long long q = (long long)floor(xd / p.M_as_double);
+        // d_k = a_k - q M_k (|d_k| < 2^46), then x - q M = sum_k d_k 2^(32 k) with signed carries
+        long long c = (long long)a0 - q * (long long)p.M[0];
+        const unsigned long long r0 = (unsigned long long)c & 0xFFFFFFFFull;
+        c = (c >> 32) + (long long)a1 - q * (long long)p.M[1];
+        const unsigned long long r1 = (unsigned long long)c & 0xFFFFFFFFull;
+        c = (c >> 32) + (long long)a2 - q * (long long)p.M[2];
+        const unsigned long long r2 = (unsigned long long)c & 0xFFFFFFFFull;
+        c = (c >> 32) + (long long)a3 - q * (long long)p.M[3];  // top limb: signed, |c| < 2^28, so its low 32 bits
+        // placed at bit 96 give the right two's-complement value even when the estimate was one too large
+        i128 x = (i128)(((u128)(unsigned long long)c << 96) | ((u128)r2 << 64) | ((u128)r1 << 32) | (u128)r0);
+        if (x < 0) x += M;
+        if (x >= M) x -= M;
+        if (x > half) x -= M;
+        out[2 * i] = (long long)(unsigned long long)(u128)x;
+        out[2 * i + 1] = (long long)(x >> 64);
+    }
+}
+
+bool build_crt_params(CrtParams* c) {
+    c->n = kNumWideModuli;
+    u128 M = 1;
+    for (int t = 0; t < kNumWideModuli; ++t) M *= (u128)kWideModuli[t];
+    for (int t = 0; t < kNumWideModuli; ++t) {
+        const int m = kWideModuli[t];
+        const u128 Mt = M / (u128)m;
+        const int mt_mod = (int)(Mt % (u128)m);
+        int inv = 0;
+        for (int a = 1; a < m && !inv; ++a)
+            if ((mt_mod * a) % m == 1) inv = a;
+        if (!inv) return false;
+        const u128 W = Mt * (u128)inv;  // < M
+        c->m[t] = m;
+        for (int k = 0; k < 4; ++k) c->w[t][k] = (unsigned int)(W >> (32 * k));
+    }
+    for (int k = 0; k < 4; ++k) c->M[k] = (unsigned int)(M >> (32 * k));
+    c->M_lo = (unsigned long long)M;
+    c->M_hi = (unsigned long long)(M >> 64);
+    c->half_lo = (unsigned long long)(M / 2);
+    c->half_hi = (unsigned long long)((M / 2) >> 64);
+    c->M_as_double = (double)c->M_hi * 18446744073709551616.0 + (double)c->M_lo;
+    return true;
+}
+
+long double log2_of_moduli_product() {
+    long double s = 0;
+    for (int t = 0; t < kNumWideModuli; ++t) s += log2l((long double)kWideModuli[t]);
+    return s;
+}
+
+struct WideLayout {
+    size_t res_a, res_b, res_c, planes, total;
+};
+
+bool wide_layout(int64_t M, int64_t N, int64_t K, WideLayout* w) {
+    size_t planes = 0;
+    for (int t = 0; t < kNumWideModuli; ++t) {
+        const size_t b = awe_workspace_bytes(AWE_ENC_MOD_M, kWideModuli[t], M, N, K);
+        if (!b) return false;
+        planes = std::max(planes, b);
+    }
+    size_t off = 0;
+    w->res_a = off;
+    off += (size_t)round_up((int64_t)kNumWideModuli * M * K, 256);
+    w->res_b = off;
+    off += (size_t)round_up((int64_t)kNumWideModuli * K * N, 256);
+    w->res_c = off;
+    off += (size_t)round_up((int64_t)kNumWideModuli * M * N * 2, 256);
+    w->planes = off;
+    off += (size_t)round_up((int64_t)planes, 256);
+    w->total = off;
+    return true;
+}
+
+}  // namespace
+
+extern "C" int awe_wide_moduli(int32_t* out, int capacity) {
+    if (out)
+        for (int t = 0; t < kNumWideModuli && t < capacity; ++t) out[t] = kWideModuli[t];
+    return kNumWideModuli;
+}
+
+extern "C" size_t awe_wide_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    WideLayout w;
+    return wide_layout(M, N, K, &w) ? w.total : 0;
+}
+
+extern "C" awe_status_t awe_wide_residues(awe_handle_t h, const int64_t* X_dev, int64_t count, int8_t* res_dev,
+                                          void* stream) {
+    if (!h || !X_dev || !res_dev || count <= 0) return AWE_ERR_INVALID_ARG;
+    if ((uintptr_t)X_dev % 16 || (uintptr_t)res_dev % 4) return AWE_ERR_ALIGNMENT;
+    ResidueParams p = {};
+    p.n = kNumWideModuli;
+    for (int t = 0; t < kNumWideModuli; ++t) {
+        const unsigned int m = (unsigned int)kWideModuli[t];
+        p.m[t] = (int)m;
+        p.c1[t] = (1u << 14) % m;
+        p.c2[t] = (1u << 28) % m;
+        p.c3[t] = (unsigned int)((1ull << 42) % m);
+        p.magic[t] = 0xFFFFFFFFu / m + 1u;
+    }
+    const long long groups = (count + 3) / 4;
+    const unsigned blocks = (unsigned)std::min<long long>((groups + 255) / 256, (long long)h->sm_count * 16);
+    wide_residues_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const long long*)X_dev, count, p, res_dev);
+    if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
+    h->launches += 1;
+    return AWE_OK;
+}
+
+extern "C" awe_status_t awe_wide_crt(awe_handle_t h, const int16_t* res_dev, int64_t count, int64_t* out_dev,
+                                     void* stream) {
+    if (!h || !res_dev || !out_dev || count <= 0) return AWE_ERR_INVALID_ARG;
+    if ((uintptr_t)res_dev % 2 || (uintptr_t)out_dev % 16) return AWE_ERR_ALIGNMENT;
+    CrtParams c = {};
+    if (!build_crt_params(&c)) return AWE_ERR_UNSUPPORTED;
+    const unsigned blocks = (unsigned)std::min<long long>((count + 255) / 256, (long long)h->sm_count * 16);
+    wide_crt_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const short*)res_dev, count, c, (long long*)out_dev);
+    if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
+    h->launches += 1;
+    return AWE_OK;
+}
+
+extern "C" awe_status_t awe_gemm_exact_wide(awe_handle_t h, const int64_t* A_dev, const int64_t* B_dev, int64_t M,
+                                            int64_t N, int64_t K, int in_bits, int64_t* C_dev, void* workspace_dev,
+                                            size_t workspace_bytes, void* stream) {
+    if (!h || !A_dev || !B_dev || !C_dev || !workspace_dev || M <= 0 || N <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
+    if (in_bits < 2 || in_bits > 54) return AWE_ERR_INVALID_ARG;
+    // unique reconstruction: prod(m) > 2 K B^2 with B = 2^(in_bits-1) - 1  (Section 5.3)
+    if (1.0L + log2l((long double)K) + 2.0L * (long double)(in_bits - 1) >= log2_of_moduli_product())
+        return AWE_ERR_RANGE;
+    WideLayout w;
+    if (!wide_layout(M, N, K, &w)) return AWE_ERR_UNSUPPORTED;
+    if (workspace_bytes < w.total) return AWE_ERR_WORKSPACE;
+    if ((uintptr_t)workspace_dev % 256 || (uintptr_t)A_dev % 16 || (uintptr_t)B_dev % 16 || (uintptr_t)C_dev % 16)
+        return AWE_ERR_ALIGNMENT;
+    uint8_t* base = (uint8_t*)workspace_dev;
+    int8_t* res_a = (int8_t*)(base + w.res_a);
+    int8_t* res_b = (int8_t*)(base + w.res_b);
+    int16_t* res_c = (int16_t*)(base + w.res_c);
+    awe_status_t s;
+    if ((s = awe_wide_residues(h, A_dev, M * K, res_a, stream)) != AWE_OK) return s;
+    if ((s = awe_wide_residues(h, B_dev, K * N, res_b, stream)) != AWE_OK) return s;
+    for (int t = 0; t < kNumWideModuli; ++t) {
+        s = awe_gemm_exact(h, res_a + (size_t)t * M * K, AWE_I8, res_b + (size_t)t * K * N, AWE_I8, M, N, K,
+                           AWE_ENC_MOD_M, kWideModuli[t], res_c + (size_t)t * M * N, AWE_C_RES_I16, base + w.planes,
+                           w.total - w.planes, stream);
+        if (s != AWE_OK) return s;
+    }
+    return awe_wide_crt(h, res_c, M * N, C_dev, stream);
+}
