@@ -238,6 +238,13 @@ awe_status_t awe_fp4_product_raw(awe_handle_t h, const void* planeX_dev, const v
  * *site (may be NULL) naming the wait that gave up.  The word is cleared by the read. */
 awe_status_t awe_last_device_status(awe_handle_t h, void* stream, int* site);
 
+/* Self-test of the failure path: launches one warp that waits, with a budget of limit_us
+ * microseconds (1 .. 1,000,000), on a barrier nothing signals.  The wait gives up, records
+ * AWE_ERR_TIMEOUT with site 1000 in the status word and the kernel returns normally; the next
+ * awe_last_device_status reports it and the handle stays usable.  Nothing faults or traps.
+ * (No counterpart in the paper.) */
+awe_status_t awe_selftest_bounded_wait(awe_handle_t h, int64_t limit_us, void* stream);
+
 /* Diagnostic: the SM clock (MHz) at which the most recent GEMM launch on this handle actually ran,
  * measured inside the kernel by CTA 0 as elapsed SM cycles over elapsed nanoseconds.  Waits for
  * `stream`.  Lets a benchmark state the tensor-pipe peak at the delivered clock (the part is

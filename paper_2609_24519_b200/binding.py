@@ -30,7 +30,7 @@ STATIC_WORKSPACE_BYTES = 24 << 20
 EXPORTS = ["awe_create", "awe_destroy", "awe_encoding_info", "awe_encoding_lut", "awe_planes_bytes",
            "awe_workspace_bytes", "awe_host_staging_bytes", "awe_encode", "awe_gemm_planes", "awe_gemm_exact",
            "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_wide_moduli", "awe_wide_workspace_bytes",
-           "awe_wide_residues", "awe_wide_crt", "awe_gemm_exact_wide", "awe_fp4_product_raw", "awe_last_device_status", "awe_last_gemm_clock_mhz", "awe_launch_count",
+           "awe_wide_residues", "awe_wide_crt", "awe_gemm_exact_wide", "awe_fp4_product_raw", "awe_last_device_status", "awe_selftest_bounded_wait", "awe_last_gemm_clock_mhz", "awe_launch_count",
            "awe_status_string"]
 
 
@@ -84,6 +84,7 @@ def lib() -> ctypes.CDLL:
     L.awe_gemm_exact_wide.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, sz, vp]
     L.awe_fp4_product_raw.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
     L.awe_last_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    L.awe_selftest_bounded_wait.argtypes = [vp, i64, vp]
     L.awe_last_gemm_clock_mhz.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
     L.awe_launch_count.argtypes = [vp]
     L.awe_launch_count.restype = i64
@@ -255,6 +256,10 @@ def awe_last_device_status(h: Handle, stream=None):
     site = ctypes.c_int(0)
     st = lib().awe_last_device_status(h.raw, _stream(stream), ctypes.byref(site))
     return int(st), int(site.value)
+
+
+def awe_selftest_bounded_wait(h: Handle, limit_us: int = 1000, stream=None) -> None:
+    _check(lib().awe_selftest_bounded_wait(h.raw, limit_us, _stream(stream)), "awe_selftest_bounded_wait")
 
 
 def awe_last_gemm_clock_mhz(h: Handle, stream=None) -> float:

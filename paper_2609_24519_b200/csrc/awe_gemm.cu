@@ -101,20 +101,42 @@ struct Shared {
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 
-__device__ __forceinline__ bool bounded_wait(Shared* sh, uint32_t bar, uint32_t parity, unsigned int* status,
-                                             int site) {
+// Wait for a phase of an mbarrier, but never for longer than limit_ns: when the budget runs out the
+// first CTA to notice records AWE_ERR_TIMEOUT and the site in the status word, every role of this
+// CTA sees the abort flag at its next poll, and the kernel winds down normally.
+__device__ __forceinline__ bool bounded_wait_ns(volatile uint32_t* abort_flag, uint32_t bar, uint32_t parity,
+                                                unsigned int* status, int site, uint64_t limit_ns) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = ptx::globaltimer_ns();
     uint32_t polls = 0;
     for (;;) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
-        if (sh->abort_flag) return false;
-        if ((++polls & 1023u) == 0 && ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
+        if (*abort_flag) return false;
+        if ((++polls & 63u) == 0 && ptx::globaltimer_ns() - t0 > limit_ns) {
             if (atomicCAS(status, 0u, (unsigned)AWE_ERR_TIMEOUT) == 0u) status[1] = (unsigned)site;
-            sh->abort_flag = 1;
+            *abort_flag = 1;
             return false;
         }
     }
+}
+
+__device__ __forceinline__ bool bounded_wait(Shared* sh, uint32_t bar, uint32_t parity, unsigned int* status,
+                                             int site) {
+    return bounded_wait_ns(&sh->abort_flag, bar, parity, status, site, kWaitLimitNs);
+}
+
+// Self-test of the bounded wait: one warp waits, with a budget of limit_ns, on a barrier that
+// nothing ever signals, so the wait must give up, record its status and let the kernel return.
+__global__ void bounded_wait_selftest_kernel(unsigned int* status, unsigned long long limit_ns, int site) {
+    __shared__ uint64_t bar;
+    __shared__ volatile uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_u32(&bar), 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    bounded_wait_ns(&abort_flag, ptx::smem_u32(&bar), 0, status, site, limit_ns);
 }
 
 __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int* tm, int* tn) {
@@ -688,6 +710,15 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
         p.accumulate = kb0 > 0;
         if ((s = launch_gemm(h, ma, mb, p, (cudaStream_t)stream)) != AWE_OK) return s;
     }
+    return AWE_OK;
+}
+
+extern "C" awe_status_t awe_selftest_bounded_wait(awe_handle_t h, int64_t limit_us, void* stream) {
+    if (!h || limit_us <= 0 || limit_us > 1000000) return AWE_ERR_INVALID_ARG;
+    bounded_wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(h->status_dev, (unsigned long long)limit_us * 1000ull,
+                                                                     1000);
+    if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
+    h->launches += 1;
     return AWE_OK;
 }
 

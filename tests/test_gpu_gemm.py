@@ -208,3 +208,24 @@ def test_argument_errors_are_reported_before_any_launch():
     with pytest.raises(b.AweError):
         b.awe_encoding_info(b.ENC_MOD_M, 170)
     assert b.awe_launch_count(h) == n0
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
+    """Failure path without a fault: a bounded wait on a barrier nothing signals gives up after its
+    budget, the kernel returns, the host reads AWE_ERR_TIMEOUT + site, and work continues."""
+    import time
+    h = b.awe_create(0)
+    t0 = time.time()
+    b.awe_selftest_bounded_wait(h, 2000)                       # 2 ms budget
+    assert b.awe_last_device_status(h) == (7, 1000)
+    assert time.time() - t0 < 5.0
+    assert b.awe_last_device_status(h) == (0, 0)               # the read cleared it
+    A, B = wl.make_inputs(wl.small("t", 128, 256, 256, seed=33))
+    ws = torch.empty(b.awe_workspace_bytes(b.ENC_INT8_AWE6, 0, 128, 256, 256), dtype=torch.uint8, device="cuda")
+    C = torch.zeros((128, 256), dtype=torch.int32, device="cuda")
+    b.awe_gemm_exact(h, torch.from_numpy(A).cuda(), b.I8, torch.from_numpy(B).cuda(), b.I8, 128, 256, 256,
+                     b.ENC_INT8_AWE6, 0, C, b.C_I32, ws)
+    torch.cuda.synchronize()
+    assert b.awe_last_device_status(h) == (0, 0)
+    assert np.array_equal(C.cpu().numpy(), mm.matmul_i64(A, B))
+    b.awe_destroy(h)
