@@ -1,5 +1,7 @@
 // Handle management and the whole-procedure entry points (Algorithm 1 end to end).
+#include <algorithm>
 #include <cstring>
+#include <initializer_list>
 #include <new>
 
 #include "awe_internal.h"
@@ -38,6 +40,14 @@ extern "C" awe_status_t awe_create(awe_handle_t* out, int device) {
 extern "C" awe_status_t awe_destroy(awe_handle_t h) {
     if (!h) return AWE_ERR_INVALID_ARG;
     cudaSetDevice(h->device);
+    if (h->copy_in) cudaStreamDestroy(h->copy_in);
+    if (h->copy_out) cudaStreamDestroy(h->copy_out);
+    for (cudaEvent_t e : {h->ev_start, h->ev_b, h->ev_done})
+        if (e) cudaEventDestroy(e);
+    for (int i = 0; i < awe_ctx::kMaxHostChunks; ++i) {
+        if (h->ev_a[i]) cudaEventDestroy(h->ev_a[i]);
+        if (h->ev_c[i]) cudaEventDestroy(h->ev_c[i]);
+    }
     if (h->status_dev) cudaFree(h->status_dev);
     if (h->lut_arena_dev) cudaFree(h->lut_arena_dev);
     delete h;
@@ -69,6 +79,8 @@ awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_i
     return AWE_OK;
 }
 }  // namespace awe
+
+static int t_planes(const awe_encoding_desc& d, awe_side_t side) { return side == AWE_SIDE_A ? d.n_planes_a : d.n_planes_b; }
 
 static size_t out_elem_bytes(awe_out_dtype_t t) { return t == AWE_C_I64 ? 8 : (t == AWE_C_RES_I16 ? 2 : 4); }
 
@@ -129,13 +141,69 @@ extern "C" awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, 
     uint8_t* dA = base + round_up((int64_t)ws, 256);
     uint8_t* dB = dA + round_up(M * K, 256);
     uint8_t* dC = dB + round_up(K * N, 256);
-    const size_t c_bytes = (size_t)M * N * out_elem_bytes(out_dt);
-    if (cudaMemcpyAsync(dA, A_host, (size_t)M * K, cudaMemcpyHostToDevice, st) != cudaSuccess) return AWE_ERR_CUDA;
-    if (cudaMemcpyAsync(dB, B_host, (size_t)K * N, cudaMemcpyHostToDevice, st) != cudaSuccess) return AWE_ERR_CUDA;
-    awe_status_t s = awe_gemm_exact(h, dA, a_dt, dB, b_dt, M, N, K, enc, modulus, dC, out_dt, base, ws, stream);
+    const size_t elem = out_elem_bytes(out_dt);
+    // Everything awe_gemm_exact would reject is rejected here, before any copy is enqueued.
+    awe_encoding_desc d;
+    awe_status_t s = awe_encoding_info(enc, modulus, &d);
     if (s != AWE_OK) return s;
-    if (cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return AWE_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return AWE_ERR_CUDA;
+    if ((d.modulus != 0) != (out_dt == AWE_C_RES_I16 || out_dt == AWE_C_RES_I32)) return AWE_ERR_UNSUPPORTED;
+    const SideTable* tbl;
+    if (!get_side_table(enc, modulus, AWE_SIDE_A, a_dt, &tbl) || !get_side_table(enc, modulus, AWE_SIDE_B, b_dt, &tbl))
+        return AWE_ERR_UNSUPPORTED;
+    const int64_t amax = std::max(std::abs(d.a_lo), std::abs(d.a_hi));
+    const int64_t bmax = std::max(std::abs(d.b_lo), std::abs(d.b_hi));
+    if (out_dt == AWE_C_I32 && (__int128)amax * bmax * K >= ((__int128)1 << 31)) return AWE_ERR_RANGE;
+
+    // Rows of A (and of C) are cut into chunks so that the copy of chunk i+1 to the device, the
+    // work on chunk i and the copy of chunk i-1 back to the host overlap (the two copy directions
+    // run on their own streams).  Small problems go through in one piece.
+    int chunks = (int)std::min<int64_t>(awe_ctx::kMaxHostChunks, M / 1024);
+    if (chunks < 2) chunks = 1;
+    if (!h->copy_in) {
+        bool ok = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&h->ev_b, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&h->ev_done, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < awe_ctx::kMaxHostChunks; ++i)
+            ok = cudaEventCreateWithFlags(&h->ev_a[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&h->ev_c[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return AWE_ERR_CUDA;
+    }
+#define AWE_CU(x) do { if ((x) != cudaSuccess) return AWE_ERR_CUDA; } while (0)
+    const int64_t pitch = plane_pitch_bytes(K);
+    uint8_t* pa = base;
+    uint8_t* pb = base + round_up((int64_t)awe_planes_bytes(enc, modulus, AWE_SIDE_A, M, K), 256);
+    AWE_CU(cudaEventRecord(h->ev_start, st));
+    AWE_CU(cudaStreamWaitEvent(h->copy_in, h->ev_start, 0));
+    AWE_CU(cudaStreamWaitEvent(h->copy_out, h->ev_start, 0));
+    AWE_CU(cudaMemcpyAsync(dB, B_host, (size_t)K * N, cudaMemcpyHostToDevice, h->copy_in));
+    AWE_CU(cudaEventRecord(h->ev_b, h->copy_in));
+    AWE_CU(cudaStreamWaitEvent(st, h->ev_b, 0));
+    if ((s = awe_encode(h, enc, modulus, AWE_SIDE_B, dB, b_dt, AWE_ROWMAJOR_KxR, N, K, N, pb, stream)) != AWE_OK) return s;
+    const int64_t rows_per_chunk = chunks == 1 ? M : round_up((M + chunks - 1) / chunks, 256);
+    int c = 0;
+    for (int64_t r0 = 0; r0 < M; r0 += rows_per_chunk, ++c) {
+        const int64_t rows = std::min(rows_per_chunk, M - r0);
+        const uint8_t* a_src = (const uint8_t*)A_host + (size_t)r0 * K;
+        uint8_t* a_dst = dA + (size_t)r0 * K;
+        uint8_t* pa_c = pa + (size_t)t_planes(d, AWE_SIDE_A) * (size_t)r0 * pitch;  // this chunk's own plane block
+        uint8_t* c_dst = dC + (size_t)r0 * N * elem;
+        AWE_CU(cudaMemcpyAsync(a_dst, a_src, (size_t)rows * K, cudaMemcpyHostToDevice, h->copy_in));
+        AWE_CU(cudaEventRecord(h->ev_a[c], h->copy_in));
+        AWE_CU(cudaStreamWaitEvent(st, h->ev_a[c], 0));
+        if ((s = awe_encode(h, enc, modulus, AWE_SIDE_A, a_dst, a_dt, AWE_ROWMAJOR_RxK, rows, K, K, pa_c, stream)) != AWE_OK)
+            return s;
+        if ((s = awe_gemm_planes(h, enc, modulus, pa_c, pb, rows, N, K, c_dst, out_dt, N, 0, stream)) != AWE_OK) return s;
+        AWE_CU(cudaEventRecord(h->ev_c[c], st));
+        AWE_CU(cudaStreamWaitEvent(h->copy_out, h->ev_c[c], 0));
+        AWE_CU(cudaMemcpyAsync((uint8_t*)C_host + (size_t)r0 * N * elem, c_dst, (size_t)rows * N * elem,
+                               cudaMemcpyDeviceToHost, h->copy_out));
+    }
+    AWE_CU(cudaEventRecord(h->ev_done, h->copy_out));
+    AWE_CU(cudaStreamWaitEvent(st, h->ev_done, 0));
+    AWE_CU(cudaStreamSynchronize(st));
+#undef AWE_CU
     return AWE_OK;
 }
 

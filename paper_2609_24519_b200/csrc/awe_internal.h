@@ -56,6 +56,12 @@ struct awe_ctx {
     std::vector<LutSlot> slots;
     int64_t launches = 0;
     void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
+    // copy engines of the host-buffer entry point: one stream per direction and the events that
+    // order them against the caller's stream (created on first use)
+    static constexpr int kMaxHostChunks = 16;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_done = nullptr;
+    cudaEvent_t ev_a[kMaxHostChunks] = {nullptr}, ev_c[kMaxHostChunks] = {nullptr};
     std::mutex mu;
 };
 

@@ -188,6 +188,35 @@ def test_host_buffer_entry_point():
     assert np.array_equal(Ch.numpy(), mm.matmul_i64(A, B))
 
 
+@pytest.mark.parametrize("enc,out_dt,tdt,modulus,kinds", [
+    (b.ENC_INT8_AWE6, b.C_I32, torch.int32, 0, ("int8", "int8")),
+    (b.ENC_INT8_AWE6, b.C_I64, torch.int64, 0, ("extreme", "extreme")),
+    (b.ENC_MOD_M, b.C_RES_I16, torch.int16, 89, ("residue", "residue")),
+])
+def test_host_buffer_entry_point_chunked(enc, out_dt, tdt, modulus, kinds):
+    """M large enough that the rows go through in several overlapped chunks (ragged last chunk)."""
+    h = gu.handle()
+    w = wl.small("t", 3300, 520, 700, kinds[0], kinds[1], seed=23, modulus=modulus)
+    A, B = wl.make_inputs(w)
+    Ah, Bh = torch.from_numpy(A).pin_memory(), torch.from_numpy(B).pin_memory()
+    Ch = torch.full((w.M, w.N), 5, dtype=tdt).pin_memory()
+    nbytes = b.awe_workspace_bytes(enc, modulus, w.M, w.N, w.K) + \
+        b.awe_host_staging_bytes(enc, modulus, w.M, w.N, w.K, out_dt)
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    want = mm.matmul_i64(A, B)
+    if modulus:
+        want = mm.mod_symmetric(want, modulus)
+    for _ in range(2):                                  # the second call reuses the handle's copy streams
+        Ch.fill_(5)
+        b.awe_gemm_exact_host(h, Ah, b.I8, Bh, b.I8, w.M, w.N, w.K, enc, modulus, Ch, out_dt, scratch)
+        assert np.array_equal(Ch.numpy().astype(np.int64), want)
+    assert b.awe_last_device_status(h) == (0, 0)
+    # pageable host memory works too
+    Cp = np.zeros((w.M, w.N), dtype=Ch.numpy().dtype)
+    b.awe_gemm_exact_host(h, A, b.I8, B, b.I8, w.M, w.N, w.K, enc, modulus, Cp, out_dt, scratch)
+    assert np.array_equal(Cp.astype(np.int64), want)
+
+
 def test_argument_errors_are_reported_before_any_launch():
     h = gu.handle()
     n0 = b.awe_launch_count(h)
