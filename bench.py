@@ -416,6 +416,38 @@ def main():
                                       "residues_GBs": 8192 * 8192 * (8 + nmod) / (ms_res * 1e-3) / 1e9,
                                       "crt_GBs": 8192 * 8192 * (2 * nmod + 16) / (ms_crt * 1e-3) / 1e9}
             del aw, bw, wsw, cw, ra, rc
+        if (M, N, K) == (8192, 8192, 8192):
+            # FP4 MMA ceiling of this kernel on this part: one raw product on all-zero planes, which
+            # draws too little power to be capped, so it shows the structural limit at ~max clock
+            kz = 65536
+            pz = torch.zeros((8192, kz // 2), dtype=torch.uint8, device=dev)
+            pzo = torch.empty((8192, 8192), dtype=torch.float32, device=dev)
+            time.sleep(1.5)                      # let the power regulator forget the runs above
+            for _ in range(100):
+                b.awe_fp4_product_raw(h, pz, pz, 8192, 8192, kz, pzo, 8192)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(10):
+                b.awe_fp4_product_raw(h, pz, pz, 8192, 8192, kz, pzo, 8192)
+            e1.record()
+            torch.cuda.synchronize()
+            ceil_tflops = 2.0 * 8192 * 8192 * kz / (e0.elapsed_time(e1) / 10 * 1e-3) / 1e12
+            ctx["fp4_ceiling_zero_data_TFLOPs"] = ceil_tflops
+            ctx["fp4_ceiling_clock_mhz"] = b.awe_last_gemm_clock_mhz(h)
+            line["roofline"]["frac_of_measured_fp4_ceiling"] = gemm_tflops / ceil_tflops
+            del pz
+            # stand-alone reconstruction (HBM pass): 6 FP32 product matrices -> int32
+            P6 = torch.zeros((6, 8192, 8192), dtype=torch.float32, device=dev)
+            for _ in range(2):
+                b.awe_reconstruct(h, enc, 0, P6, 8192 * 8192, 8192, 8192, 8192, pzo, b.C_I32, 8192)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(5):
+                b.awe_reconstruct(h, enc, 0, P6, 8192 * 8192, 8192, 8192, 8192, pzo, b.C_I32, 8192)
+            e1.record()
+            torch.cuda.synchronize()
+            ctx["standalone_reconstruct_GBs"] = 8192 * 8192 * 28 / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e9
+            del P6, pzo
         ctx["paper_theoretical_TOPS"] = "1500 (9.0 PFLOPS / 6, published peak, not a measurement; B200)"
         line["context"] = ctx
 

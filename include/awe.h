@@ -237,6 +237,16 @@ awe_status_t awe_gemm_exact_static(const void* A_dev, awe_in_dtype_t a_dt, const
 awe_status_t awe_fp4_product_raw(awe_handle_t h, const void* planeX_dev, const void* planeY_dev, int64_t M,
                                  int64_t N, int64_t K, float* P_dev, int64_t ldp, void* stream);
 
+/* Stand-alone reconstruction (Algorithm 1, last step; Section 5.3 for the residue form) from the r
+ * raw FP32 products of an encoding, e.g. written by awe_fp4_product_raw: product k is the M x N
+ * matrix at P_dev + k * plane_stride with leading dimension ldp (floats, doubled-integer
+ * convention).  Writes C = (sum_k l_k P_k) >> log2 D, or that sum mod m in the symmetric range, to
+ * C_dev (leading dimension ldc, type out_dt).  The unfused counterpart of the epilogue of
+ * awe_gemm_planes; every P_k must come from a single exact accumulation segment (K <= K*). */
+awe_status_t awe_reconstruct(awe_handle_t h, int enc, int modulus, const float* P_dev, int64_t plane_stride,
+                             int64_t ldp, int64_t M, int64_t N, void* C_dev, awe_out_dtype_t out_dt, int64_t ldc,
+                             void* stream);
+
 /* Wait for `stream` and read the handle's device status word: AWE_OK, or AWE_ERR_TIMEOUT with
  * *site (may be NULL) naming the wait that gave up.  The word is cleared by the read. */
 awe_status_t awe_last_device_status(awe_handle_t h, void* stream, int* site);

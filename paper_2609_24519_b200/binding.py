@@ -30,7 +30,7 @@ STATIC_WORKSPACE_BYTES = 24 << 20
 EXPORTS = ["awe_create", "awe_destroy", "awe_encoding_info", "awe_encoding_lut", "awe_planes_bytes",
            "awe_workspace_bytes", "awe_host_staging_bytes", "awe_encode", "awe_gemm_planes", "awe_gemm_exact",
            "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_wide_moduli", "awe_wide_workspace_bytes",
-           "awe_wide_residues", "awe_wide_crt", "awe_gemm_exact_wide", "awe_fp4_product_raw", "awe_last_device_status", "awe_selftest_bounded_wait", "awe_last_gemm_clock_mhz", "awe_launch_count",
+           "awe_wide_residues", "awe_wide_crt", "awe_gemm_exact_wide", "awe_reconstruct", "awe_fp4_product_raw", "awe_last_device_status", "awe_selftest_bounded_wait", "awe_last_gemm_clock_mhz", "awe_launch_count",
            "awe_status_string"]
 
 
@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
     L.awe_wide_residues.argtypes = [vp, vp, i64, vp, vp]
     L.awe_wide_crt.argtypes = [vp, vp, i64, vp, vp]
     L.awe_gemm_exact_wide.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, sz, vp]
+    L.awe_reconstruct.argtypes = [vp, i32, i32, vp, i64, i64, i64, i64, vp, i32, i64, vp]
     L.awe_fp4_product_raw.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
     L.awe_last_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.awe_selftest_bounded_wait.argtypes = [vp, i64, vp]
@@ -250,6 +251,12 @@ def awe_gemm_exact_wide(h: Handle, A, B, M: int, N: int, K: int, in_bits: int, C
 def awe_fp4_product_raw(h: Handle, planeX, planeY, M: int, N: int, K: int, P, ldp: int, stream=None) -> None:
     _check(lib().awe_fp4_product_raw(h.raw, _ptr(planeX), _ptr(planeY), M, N, K, _ptr(P), ldp, _stream(stream)),
            "awe_fp4_product_raw")
+
+
+def awe_reconstruct(h: Handle, enc: int, modulus: int, P, plane_stride: int, ldp: int, M: int, N: int, C,
+                    out_dt: int, ldc: int, stream=None) -> None:
+    _check(lib().awe_reconstruct(h.raw, enc, modulus, _ptr(P), plane_stride, ldp, M, N, _ptr(C), out_dt, ldc,
+                                 _stream(stream)), "awe_reconstruct")
 
 
 def awe_last_device_status(h: Handle, stream=None):

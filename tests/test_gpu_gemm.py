@@ -168,6 +168,38 @@ def test_planes_entry_with_leading_dimension_and_guard_columns():
         assert np.all(got[:, 200:] == 77)                  # nothing written past N
 
 
+@pytest.mark.parametrize("enc,modulus,out_dt,kinds", [
+    (b.ENC_INT8_AWE6, 0, b.C_I32, ("int8", "int8")),
+    (b.ENC_INT8_BASE13_9, 0, b.C_I64, ("extreme", "extreme")),
+    (b.ENC_INT4xINT8_AWE4, 0, b.C_I32, ("int4", "int8")),
+    (b.ENC_MOD_M, 89, b.C_RES_I16, ("residue", "residue")),
+])
+def test_unfused_products_plus_standalone_reconstruction_equal_the_fused_kernel(enc, modulus, out_dt, kinds):
+    """Algorithm 1 with its steps apart: every product k as a raw FP32 matrix (one FP4 GEMM each),
+    then the stand-alone reconstruction -- must equal the fused kernel and the oracle."""
+    h = gu.handle()
+    w = wl.small("t", 200, 333, 900, kinds[0], kinds[1], seed=27, modulus=modulus)
+    A, B = wl.make_inputs(w)
+    d = b.awe_encoding_info(enc, modulus)
+    a_dt = b.I4_IN_I8 if enc == b.ENC_INT4xINT8_AWE4 else b.I8
+    pa = gu.gpu_encode(enc, modulus, b.SIDE_A, A, a_dt)
+    pb = gu.gpu_encode(enc, modulus, b.SIDE_B, np.ascontiguousarray(B.T))
+    dpa, dpb = torch.from_numpy(pa).cuda(), torch.from_numpy(pb).cuda()
+    ldp = 336
+    P = torch.zeros((d.r, w.M, ldp), dtype=torch.float32, device="cuda")
+    for k in range(d.r):
+        b.awe_fp4_product_raw(h, dpa[d.ia[k]], dpb[d.ib[k]], w.M, w.N, w.K, P[k], ldp)
+    C = torch.full((w.M, w.N), 9, dtype=gu.TORCH_OUT[out_dt], device="cuda")
+    b.awe_reconstruct(h, enc, modulus, P, w.M * ldp, ldp, w.M, w.N, C, out_dt, w.N)
+    torch.cuda.synchronize()
+    want = mm.matmul_i64(A, B)
+    if modulus:
+        want = mm.mod_symmetric(want, modulus)
+    assert np.array_equal(C.cpu().numpy().astype(np.int64), want)
+    fused = gu.gpu_gemm_exact(A, B, enc, out_dt, modulus=modulus, a_dt=a_dt)
+    assert np.array_equal(fused, C.cpu().numpy())
+
+
 def test_results_are_reproducible_run_to_run():
     A, B = wl.make_inputs(wl.small("t", 512, 768, 2048, seed=31))
     first = gu.gpu_gemm_exact(A, B, b.ENC_INT8_AWE6, b.C_I32)
