@@ -58,8 +58,10 @@ typedef enum {
     AWE_ENC_INT4xINT8_AWE4 = 3, /* INT4xINT8, 4 products, D = 2               (Appendix A)             */
     AWE_ENC_MOD_M = 4,          /* residue form mod `modulus`, 1/3/4 products (Section 5.3)            */
     AWE_ENC_INT8_AWE6_ALT = 5,  /* INT8xINT8, 6 products, w = v = (1,11,39)   (Section 4.3)            */
-    AWE_ENC_TERNARY_INT8_3 = 6  /* {0,+-1}xINT8, 3 products: one limb against the three base-13 limbs
+    AWE_ENC_TERNARY_INT8_3 = 6, /* {0,+-1}xINT8, 3 products: one limb against the three base-13 limbs
                                    (Section 6.2), K* = 2,097,152                                       */
+    AWE_ENC_INT4xINT4_3 = 7     /* INT4xINT4, 3 products (count from Section 5.2; the encoding is not
+                                   printed: planes a0, a1, a0-a1 with weights (1,3))                  */
 } awe_encoding_t;
 
 typedef enum {

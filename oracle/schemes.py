@@ -209,6 +209,14 @@ TERNARY3 = Scheme("ternary_x_int8_3", (1,), (1, 13, 169),
                   ((1,), (1,), (1,)), tuple(_unit(j, 3) for j in range(3)), (1, 13, 169))
 
 
+# Section 5.2 states that INT4xINT4 takes 3 products but does not print the encoding.  Construction
+# used here: the Karatsuba-type step on the (2,2) cell with planes (a0, a1, a0 - a1),
+#   xy = (1 + w1) a0 b0 + (w1^2 + w1) a1 b1 - w1 (a0 - a1)(b0 - b1),
+# with w1 = 3, the weight whose tables need the smallest plane values (|plane| <= 2, coverage 16).
+INT4X4_3 = Scheme("int4xint4_3", (1, 3), (1, 3), ((1, 0), (0, 1), (1, -1)), ((1, 0), (0, 1), (1, -1)),
+                  (4, 12, -3))
+
+
 def _fp16_m12() -> Scheme:
     """Appendix A, "FP16xFP16 in 12 products": w = (1, 9, 71, 639),
     2AB = sum_{k,l} 71^(k+l) (-7 P[2k,2l] + 126 P[2k+1,2l+1] + 9 Q[k,l])."""

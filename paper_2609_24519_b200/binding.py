@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libawe_b200.so")
 OK = 0
 ENC_INT8_AWE6, ENC_INT8_BASE13_9, ENC_INT4xINT8_AWE4, ENC_MOD_M, ENC_INT8_AWE6_ALT = 1, 2, 3, 4, 5
 ENC_TERNARY_INT8_3 = 6
+ENC_INT4xINT4_3 = 7
 I8, I4_IN_I8, T2_IN_I8 = 0, 1, 2
 C_I32, C_I64, C_RES_I16, C_RES_I32 = 0, 1, 2, 3
 SIDE_A, SIDE_B = 0, 1

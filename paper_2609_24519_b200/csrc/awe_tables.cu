@@ -103,6 +103,23 @@ Scheme make_ternary() {
     return s;
 }
 
+Scheme make_int4x4() {
+    // x = a0 + 3 a1 on both sides, planes (a0, a1, a0 - a1):
+    //   xy = (1 + 3) a0 b0 + (9 + 3) a1 b1 - 3 (a0 - a1)(b0 - b1)
+    Scheme s;
+    s.p = s.q = 2;
+    s.r = 3;
+    set_vec(s.w, {1, 3});
+    set_vec(s.v, {1, 3});
+    const int pl[3][2] = {{1, 0}, {0, 1}, {1, -1}};
+    for (int k = 0; k < 3; ++k)
+        for (int i = 0; i < 2; ++i) s.alpha[k][i] = s.beta[k][i] = pl[k][i];
+    set_vec(s.ell, {4, 12, -3});
+    s.a_lo = s.b_lo = -8;
+    s.a_hi = s.b_hi = 7;
+    return s;
+}
+
 struct Choice {
     int max_abs, sum_abs;
     int limbs[kMaxLimbs];
@@ -261,6 +278,7 @@ std::map<std::tuple<int, int, int, int>, SideTable> g_tables;
 
 awe_in_dtype_t natural_dtype(int enc, awe_side_t side) {
     if (enc == AWE_ENC_INT4xINT8_AWE4 && side == AWE_SIDE_A) return AWE_I4_IN_I8;
+    if (enc == AWE_ENC_INT4xINT4_3) return AWE_I4_IN_I8;
     if (enc == AWE_ENC_TERNARY_INT8_3 && side == AWE_SIDE_A) return AWE_T2_IN_I8;
     return AWE_I8;
 }
@@ -291,6 +309,10 @@ bool get_scheme(int enc, int modulus, Scheme* out) {
             break;
         case AWE_ENC_INT4xINT8_AWE4:
             s = make_awe4();
+            ok = true;
+            break;
+        case AWE_ENC_INT4xINT4_3:
+            s = make_int4x4();
             ok = true;
             break;
         case AWE_ENC_TERNARY_INT8_3:

@@ -100,6 +100,13 @@ def test_int4_x_int8():
         assert np.array_equal(got, mm.matmul_i64(A, B))
 
 
+def test_int4_x_int4_three_products():
+    for (M, N, K) in [(256, 512, 1024), (130, 270, 300)]:
+        A, B = wl.make_inputs(wl.small("t", M, N, K, "int4", "int4", seed=29))
+        got = gu.gpu_gemm_exact(A, B, b.ENC_INT4xINT4_3, b.C_I32, a_dt=b.I4_IN_I8, b_dt=b.I4_IN_I8)
+        assert np.array_equal(got, mm.matmul_i64(A, B))
+
+
 def test_ternary_x_int8():
     """Section 6.2: {0, +-1} x INT8 in 3 products (one limb against the three base-13 limbs)."""
     for (M, N, K) in [(256, 512, 1024), (130, 270, 300), (1, 1, 1)]:

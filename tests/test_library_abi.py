@@ -41,6 +41,10 @@ def test_records_match_the_paper_and_the_oracle(b):
     s = sc.TERNARY3
     assert d.r == 3 and list(d.ell)[:3] == list(s.ell) and list(d.ib)[:3] == s.plane_index("B")
     assert (d.n_planes_a, d.n_planes_b, d.c_a, d.c_b, d.k_star) == (1, 3, 1, 8, 2097152)
+    d = b.awe_encoding_info(b.ENC_INT4xINT4_3)
+    assert d.r == 3 and list(d.ell)[:3] == list(sc.INT4X4_3.ell) and (d.c_a, d.c_b, d.k_star) == (2, 2, 4194304)
+    lut = b.awe_encoding_lut(b.ENC_INT4xINT4_3, 0, b.SIDE_B, b.I4_IN_I8)
+    assert np.array_equal(lut[np.arange(-8, 8) & 0xFF], pl.plane_lut(sc.INT4X4_3, "B", -8, 7))
     d = b.awe_encoding_info(b.ENC_INT8_AWE6)
     assert (d.c_a, d.c_b, d.k_star) == (6, 6, 466033)
     d = b.awe_encoding_info(b.ENC_INT4xINT8_AWE4)

@@ -70,7 +70,7 @@ def test_awe6_scalar_coefficient_relations():
     assert (l["P01"], l["P02"], l["P12"]) == (29, 37, 29 * 37)
 
 
-@pytest.mark.parametrize("s", [sc.AWE6, sc.AWE6_ALT, sc.AWE4, sc.BASE13_9, sc.TERNARY3, sc.FP16_M12],
+@pytest.mark.parametrize("s", [sc.AWE6, sc.AWE6_ALT, sc.AWE4, sc.BASE13_9, sc.TERNARY3, sc.INT4X4_3, sc.FP16_M12],
                          ids=lambda s: s.name)
 def test_matrix_identity(s):
     assert sc.coefficient_identity_holds(s)
@@ -126,6 +126,20 @@ def test_all_256x256_int8_pairs(s):
 
 def test_all_int4_x_int8_pairs():
     _all_pairs(sc.AWE4, list(range(-8, 8)), list(range(-128, 128)))
+
+
+def test_int4_x_int4_in_three_products():
+    # the count is the paper's (Section 5.2); the encoding is this oracle's construction
+    s = sc.INT4X4_3
+    assert s.r == 3 and sc.coefficient_identity_holds(s)
+    _all_pairs(s, list(range(-8, 8)), list(range(-8, 8)))
+    t = sc.value_table(s.w, s.alpha)
+    assert sc.coverage(t) == 16
+    assert pl.scheme_constants(s, (-8, 7), (-8, 7)) == {"c_A": 2, "c_B": 2, "K_star": 4194304}
+    # w1 = 3 is the weight with the smallest plane values among those that cover [-8, 7]
+    best = min((max(abs(sc.dot(p, sc.value_table((1, w), s.alpha)[x])) for x in range(-8, 8) for p in s.alpha), w)
+               for w in range(2, 8) if sc.coverage(sc.value_table((1, w), s.alpha)) >= 8)
+    assert best == (2, 3)
 
 
 def test_all_ternary_x_int8_pairs():
