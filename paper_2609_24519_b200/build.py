@@ -8,7 +8,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(os.path.dirname(PKG), "include")
 LIB = os.path.join(PKG, "libawe_b200.so")
-SOURCES = ["awe_tables.cu", "awe_encode.cu", "awe_gemm.cu", "awe_api.cu", "awe_static.cu", "awe_wide.cu", "awe_reconstruct.cu"]
+SOURCES = ["awe_tables.cu", "awe_encode.cu", "awe_gemm.cu", "awe_gemm_wide.cu", "awe_api.cu", "awe_static.cu", "awe_wide.cu", "awe_reconstruct.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
 

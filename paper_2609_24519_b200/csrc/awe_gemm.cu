@@ -27,17 +27,13 @@
 #include <cstdio>
 #include <cstdlib>
 
-#include "awe_internal.h"
-#include "ptx.cuh"
+#include "gemm_common.cuh"
 
 namespace awe {
+using namespace gemm;
 namespace {
 
-constexpr int kTileM = 128;  // rows of A (and of the accumulator) per CTA
 constexpr int kTileN = 256;
-constexpr int kBlockKBytes = 128;  // 256 E2M1 elements: one 128-byte swizzle row
-constexpr int kABytes = kTileM * kBlockKBytes;  // 16 KB
-
 #ifndef AWE_PAIR_STAGES
 #define AWE_PAIR_STAGES 6
 #endif
@@ -55,39 +51,12 @@ struct Cfg {
                                        ((uint32_t)((kTileM * kCtas) >> 4) << 24);
 };
 constexpr int kMaxStages = 7;
-constexpr int kThreads = 320;
-constexpr int kEpiWarps = 8;
-constexpr int kStageWarpBytes = 4096;  // 32 rows x 128 bytes per epilogue warp for the write-out
-constexpr uint32_t kTmemCols = 512;
 // Two accumulators of 256 columns and 32 columns of scale bytes do not fit 512 columns side by
 // side, so accumulator 1 starts inside the last 32 columns of accumulator 0.  The epilogue reads
 // those shared columns first and releases them separately (overlap_free), which lets the MMAs of
 // the next segment start while the rest of the previous accumulator is still being drained.
 constexpr uint32_t kAccCol0 = 0;
 constexpr uint32_t kAccCol1 = 224;
-constexpr uint32_t kSfaCol = 480;  // 16 columns of constant scale bytes each for A and B
-constexpr uint32_t kSfbCol = 496;
-
-enum OutMode { OUT_I32 = 0, OUT_I64 = 1, OUT_RES_I16 = 2, OUT_RES_I32 = 3, OUT_RAW_F32 = 4 };
-
-struct GemmParams {
-    int M, N;
-    int tiles_m, tiles_n;
-    int kblock0;        // first 256-element K block of this launch
-    int num_kblocks;    // K blocks of this launch
-    int chunk_kblocks;  // K blocks per exact accumulation segment
-    int r;
-    int ia[AWE_MAX_PRODUCTS], ib[AWE_MAX_PRODUCTS], ell[AWE_MAX_PRODUCTS];
-    int log2D, modulus;
-    int out_mode, accumulate;
-    void* C;
-    long long ldc;
-    unsigned int* status;
-    unsigned long long* clock_probe;  // [0] SM cycles, [1] nanoseconds spent by CTA 0 in this launch
-    int vec_store;     // C rows are 16-byte aligned: vector stores allowed
-    float acc_scale;   // accumulator value -> product of doubled integers
-    uint32_t sf_word;  // four copies of the UE8M0 scale byte
-};
 
 struct Shared {
     uint64_t full[kMaxStages];
@@ -99,26 +68,6 @@ struct Shared {
     volatile uint32_t abort_flag;
 };
 
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
-
-// Wait for a phase of an mbarrier, but never for longer than limit_ns: when the budget runs out the
-// first CTA to notice records AWE_ERR_TIMEOUT and the site in the status word, every role of this
-// CTA sees the abort flag at its next poll, and the kernel winds down normally.
-__device__ __forceinline__ bool bounded_wait_ns(volatile uint32_t* abort_flag, uint32_t bar, uint32_t parity,
-                                                unsigned int* status, int site, uint64_t limit_ns) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = ptx::globaltimer_ns();
-    uint32_t polls = 0;
-    for (;;) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if ((++polls & 63u) == 0 && ptx::globaltimer_ns() - t0 > limit_ns) {
-            if (atomicCAS(status, 0u, (unsigned)AWE_ERR_TIMEOUT) == 0u) status[1] = (unsigned)site;
-            *abort_flag = 1;
-            return false;
-        }
-    }
-}
 
 __device__ __forceinline__ bool bounded_wait(Shared* sh, uint32_t bar, uint32_t parity, unsigned int* status,
                                              int site) {
@@ -139,21 +88,6 @@ __global__ void bounded_wait_selftest_kernel(unsigned int* status, unsigned long
     bounded_wait_ns(&abort_flag, ptx::smem_u32(&bar), 0, status, site, limit_ns);
 }
 
-__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int* tm, int* tn) {
-    constexpr int kGroupM = 8;
-    const int per_group = kGroupM * tiles_n;
-    const int group = t / per_group, in_group = t % per_group;
-    const int first_m = group * kGroupM;
-    const int gsize = min(tiles_m - first_m, kGroupM);
-    *tm = first_m + in_group % gsize;
-    *tn = in_group / gsize;
-}
-
-// Order of the products inside a tile: ascending on a worker's even tiles, descending on its odd
-// ones, so the planes used last by one tile are the first the next tile asks L2 for.  The sum of
-// the products does not depend on the order.
-__device__ __forceinline__ int product_at(int kk, int tile_iter, int r) { return (tile_iter & 1) ? r - 1 - kk : kk; }
-
 // Residue arithmetic in FP32 (Section 5.3).  Every quantity is an integer of magnitude below 2^22
 // held exactly in a float; x mod m is taken without leaving the FP32 pipe: q = round(x / m) by the
 // add-and-subtract-1.5*2^23 trick, r = x - q m by one exact FMA, and one correction step in each
@@ -173,17 +107,6 @@ struct EpiMath {
     float mf, inv_m, lo, hi;  // modulus and its symmetric range as floats
     int reduce_each;          // reduce the running residue sum after every segment (very long K only)
 };
-
-// All lanes of the warp have finished reading their TMEM columns: one arrival for the warp on a
-// barrier of this CTA or, in a pair, of CTA 0 (cluster address).
-__device__ __forceinline__ void release(uint32_t bar, int lane, bool remote) {
-    ptx::tc_fence_before();
-    __syncwarp();
-    if (lane == 0) {
-        if (remote) ptx::mbar_arrive_cluster(bar);
-        else ptx::mbar_arrive(bar);
-    }
-}
 
 // Drain 32 accumulator columns (block BLK of this thread's 128) and fold them into the running sums.
 // When `early_bar` is non-zero these are the columns the two accumulators share: they are handed
@@ -220,56 +143,6 @@ __device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128]
         for (int i = 0; i < 32; ++i)
             sum[BLK * 32 + i] += (uint32_t)ell * (uint32_t)__float2int_rn(__uint_as_float(v[i]) * em.acc_scale);
     }
-}
-
-// Write 32 rows x 128 bytes held one row per lane (chunk(c), c = 0..7, yields its 16-byte pieces) to global memory through a
-// 4 KB shared-memory block (16-byte chunks XOR-swizzled by row so neither pass has bank conflicts):
-// afterwards lane l holds chunk l%8 of rows l/8, l/8+4, ... and one store instruction covers 4 rows
-// x 128 contiguous bytes.  bytes_valid (<= 128, may be <= 0) is how much of the row piece lies
-// inside the matrix; pieces that are cut or rows that are not 16-byte aligned fall back to
-// element-wise stores.  With `add64` the 8-byte elements are added to what is already there.
-template <int elem, class ChunkFn>
-__device__ __forceinline__ void store_rows_128b(uint8_t* stage, int lane, ChunkFn chunk, uint8_t* gbase,
-                                                long long row_pitch, int rows_valid, int bytes_valid, int vec_ok,
-                                                bool add64) {
-    if (bytes_valid <= 0 || rows_valid <= 0) return;  // warp-uniform
-#pragma unroll
-    for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) = chunk(c);
-    __syncwarp();
-    const int c = lane & 7;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int r = i * 4 + (lane >> 3);
-        const uint4 v = *reinterpret_cast<const uint4*>(stage + r * 128 + ((c ^ (r & 7)) << 4));
-        if (r >= rows_valid) continue;
-        uint8_t* dst = gbase + r * row_pitch + c * 16;
-        if (vec_ok && c * 16 + 16 <= bytes_valid) {
-            if (add64) {
-                const longlong2 old = *reinterpret_cast<const longlong2*>(dst);
-                const long long a = (long long)(((unsigned long long)v.y << 32) | v.x) + old.x;
-                const long long b = (long long)(((unsigned long long)v.w << 32) | v.z) + old.y;
-                *reinterpret_cast<longlong2*>(dst) = make_longlong2(a, b);
-            } else {
-                *reinterpret_cast<uint4*>(dst) = v;
-            }
-        } else {
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int e = 0; e < 16 / elem; ++e) {
-                if (c * 16 + (e + 1) * elem > bytes_valid) continue;
-                if (elem == 4) {
-                    reinterpret_cast<uint32_t*>(dst)[e] = w[e];
-                } else if (elem == 2) {
-                    reinterpret_cast<uint16_t*>(dst)[e] = (uint16_t)(w[e >> 1] >> (16 * (e & 1)));
-                } else {
-                    const long long x = (long long)(((unsigned long long)w[2 * e + 1] << 32) | w[2 * e]);
-                    long long* d = reinterpret_cast<long long*>(dst) + e;
-                    *d = add64 ? *d + x : x;
-                }
-            }
-        }
-    }
-    __syncwarp();
 }
 
 template <bool kPair>
@@ -568,25 +441,6 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// planes: n_planes x rows x pitch bytes.  Box: 128 bytes of K x box_rows rows of one plane.
-awe_status_t make_plane_map(awe_ctx* h, const void* planes, int64_t rows, int64_t pitch, int n_planes,
-                            int box_rows, CUtensorMap* out) {
-    if (!h->encode_tiled) return AWE_ERR_CUDA;
-    cuuint64_t dims[3] = {(cuuint64_t)pitch, (cuuint64_t)rows, (cuuint64_t)n_planes};
-    cuuint64_t strides[2] = {(cuuint64_t)pitch, (cuuint64_t)pitch * (cuuint64_t)rows};
-    cuuint32_t box[3] = {(cuuint32_t)kBlockKBytes, (cuuint32_t)box_rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = ((EncodeTiledFn)h->encode_tiled)(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(planes),
-                                                  dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? AWE_OK : AWE_ERR_CUDA;
-}
-
 // The pair variant is the default; AWE_GEMM_SINGLE_CTA=1 in the environment selects the other.
 bool use_pairs() {
     static const bool v = [] {
@@ -670,9 +524,15 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
     if (out_dt == AWE_C_I32 && (__int128)amax * bmax * K >= ((__int128)1 << 31)) return AWE_ERR_RANGE;
 
     const int64_t pitch = plane_pitch_bytes(K);
+    // 64-bit running sums are needed when not even one 256-element K block keeps D*C within 32 bits
+    static const bool force_wide = [] { const char* e = getenv("AWE_FORCE_WIDE_SUMS"); return e && e[0] == '1'; }();
+    const bool wide = !residue && (force_wide || ((int64_t)1 << 30) / (amax * bmax * ((int64_t)1 << d.log2D)) < 256);
+    if (wide && !use_pairs()) return AWE_ERR_UNSUPPORTED;
     CUtensorMap ma, mb;
     if ((s = make_plane_map(h, planesA_dev, M, pitch, d.n_planes_a, kTileM, &ma)) != AWE_OK) return s;
-    if ((s = make_plane_map(h, planesB_dev, N, pitch, d.n_planes_b, b_box_rows(), &mb)) != AWE_OK) return s;
+    if ((s = make_plane_map(h, planesB_dev, N, pitch, d.n_planes_b, wide ? wide_b_box_rows() : b_box_rows(), &mb)) !=
+        AWE_OK)
+        return s;
 
     GemmParams p = {};
     p.M = (int)M;
@@ -697,6 +557,12 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
     if (residue) kc = std::min<int64_t>(kc, std::max<int64_t>(256, d.k_star / 4 / 256 * 256));
     p.chunk_kblocks = (int)std::min<int64_t>(kc / 256, 1 << 20);
     const int64_t total_kblocks = pitch / kBlockKBytes;
+    if (wide) {
+        p.kblock0 = 0;
+        p.num_kblocks = (int)total_kblocks;
+        p.accumulate = 0;
+        return launch_gemm_wide(h, ma, mb, p, (cudaStream_t)stream);
+    }
     // 64-bit results: K is cut into launches whose own result fits 32 bits, added in int64
     int64_t seg_kblocks = total_kblocks;
     if (out_dt == AWE_C_I64 && !residue) {
