@@ -370,6 +370,22 @@ def main():
                        16384)
             ctx["worst_case_4096x4096x16384_int64_TOPS"] = 2.0 * 4096 * 4096 * 16384 / (ms * 1e-3) / 1e12
             del ax, bx
+            # width-12 integers (FP16 significands), 12 products, 64-bit reconstruction
+            a12 = torch.randint(-2047, 2048, (8192, 8192), dtype=torch.int16, device=dev, generator=gen)
+            b12 = torch.randint(-2047, 2048, (8192, 8192), dtype=torch.int16, device=dev, generator=gen)
+            ws12 = torch.empty(b.awe_workspace_bytes(b.ENC_FP16SIG_AWE12, 0, 8192, 8192, 8192), dtype=torch.uint8,
+                               device=dev)
+            c12 = torch.empty((8192, 8192), dtype=torch.int64, device=dev)
+            for _ in range(2):
+                b.awe_gemm_exact(h, a12, b.I16, b12, b.I16, 8192, 8192, 8192, b.ENC_FP16SIG_AWE12, 0, c12, b.C_I64, ws12)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(3):
+                b.awe_gemm_exact(h, a12, b.I16, b12, b.I16, 8192, 8192, 8192, b.ENC_FP16SIG_AWE12, 0, c12, b.C_I64, ws12)
+            e1.record()
+            torch.cuda.synchronize()
+            ctx["fp16_significand_awe12_8192_TOPS"] = ops / (e0.elapsed_time(e1) / 3 * 1e-3) / 1e12
+            del a12, b12, ws12, c12
             from oracle.rns import RNS_SET_FP64   # the list of moduli only (a constant, no arithmetic)
             total_ms, prods = 0.0, 0
             for m_ in RNS_SET_FP64:

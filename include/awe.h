@@ -60,14 +60,19 @@ typedef enum {
     AWE_ENC_INT8_AWE6_ALT = 5,  /* INT8xINT8, 6 products, w = v = (1,11,39)   (Section 4.3)            */
     AWE_ENC_TERNARY_INT8_3 = 6, /* {0,+-1}xINT8, 3 products: one limb against the three base-13 limbs
                                    (Section 6.2), K* = 2,097,152                                       */
-    AWE_ENC_INT4xINT4_3 = 7     /* INT4xINT4, 3 products (count from Section 5.2; the encoding is not
+    AWE_ENC_INT4xINT4_3 = 7,    /* INT4xINT4, 3 products (count from Section 5.2; the encoding is not
                                    printed: planes a0, a1, a0-a1 with weights (1,3))                  */
+    AWE_ENC_FP16SIG_AWE12 = 8   /* width-12 integers (FP16 significands with sign, |x| <= 2047; the
+                                   table also covers -2048), 12 products, w = v = (1,9,71,639), D = 2
+                                   (Appendix A).  16-bit inputs (AWE_I16); 64-bit reconstruction.     */
 } awe_encoding_t;
 
 typedef enum {
     AWE_I8 = 0,      /* one signed 8-bit value per byte                                          */
     AWE_I4_IN_I8 = 1, /* one signed 4-bit value per byte; only the low nibble is read (sign-extended) */
-    AWE_T2_IN_I8 = 2  /* one ternary value -1, 0 or +1 per byte; any other byte is read as 0         */
+    AWE_T2_IN_I8 = 2, /* one ternary value -1, 0 or +1 per byte; any other byte is read as 0         */
+    AWE_I16 = 3       /* one signed 12-bit value per 16-bit element; only the low 12 bits are read
+                         (sign-extended).  Leading dimensions stay in elements.                      */
 } awe_in_dtype_t;
 
 typedef enum {
@@ -115,7 +120,8 @@ awe_status_t awe_encoding_info(int enc, int modulus, awe_encoding_desc* out);
 
 /* Decomposition table of one side (first two loops of Algorithm 1), host only: for every
  * raw input byte b (index b & 0xFF, interpreted per `dt`) the n_planes stored plane values,
- * lut_host[256 * n_planes], row b.  Used to compare the table against an independent one. */
+ * lut_host[256 * n_planes], row b; for AWE_I16 the index is the low 12 bits of the element and the
+ * table has 4096 rows.  Used to compare the table against an independent one. */
 awe_status_t awe_encoding_lut(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, int8_t* lut_host);
 
 /* Bytes of the packed-plane buffer of one operand: n_planes x R x pitch, pitch =

@@ -35,6 +35,7 @@ def _load():
         _lib.oracle_matmul_i64.argtypes = [p, p, p, i64, i64, i64]
         _lib.oracle_matmul_i64_rows.argtypes = [p, p, p, i64, i64, i64, i64]
         _lib.oracle_mod_symmetric.argtypes = [p, i64, i64]
+        _lib.oracle_matmul_i64_s16_rows.argtypes = [p, p, p, i64, i64, i64, i64]
         _lib.oracle_threads.restype = ctypes.c_int
     return _lib
 
@@ -68,6 +69,18 @@ def matmul_i64_rows(A: np.ndarray, B: np.ndarray, i0: int, i1: int) -> np.ndarra
     assert 0 <= i0 <= i1 <= M
     C = np.empty((i1 - i0, N), dtype=np.int64)
     _load().oracle_matmul_i64_rows(A.ctypes.data, B.ctypes.data, C.ctypes.data, i0, i1, N, K)
+    return C
+
+
+def matmul_i64_s16(A: np.ndarray, B: np.ndarray, i0: int = 0, i1: int = None) -> np.ndarray:
+    """Rows i0..i1-1 (default: all) of the exact product of int16 matrices, int64."""
+    A, B = np.ascontiguousarray(A), np.ascontiguousarray(B)
+    assert A.dtype == np.int16 and B.dtype == np.int16 and A.shape[1] == B.shape[0]
+    M, K = A.shape
+    N = B.shape[1]
+    i1 = M if i1 is None else i1
+    C = np.empty((i1 - i0, N), dtype=np.int64)
+    _load().oracle_matmul_i64_s16_rows(A.ctypes.data, B.ctypes.data, C.ctypes.data, i0, i1, N, K)
     return C
 
 

@@ -62,3 +62,19 @@ void oracle_mod_symmetric(int64_t* C, int64_t count, int64_t m)
         C[t] = x + lo;
     }
 }
+
+/* The same definition for 16-bit inputs (the width-12 significand products). */
+void oracle_matmul_i64_s16_rows(const int16_t* A, const int16_t* B, int64_t* C_rows, int64_t i0, int64_t i1, int64_t N,
+                                int64_t K)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = i0; i < i1; ++i) {
+        int64_t* c = C_rows + (i - i0) * N;
+        memset(c, 0, (size_t)N * sizeof(int64_t));
+        for (int64_t k = 0; k < K; ++k) {
+            const int64_t a = A[i * K + k];
+            const int16_t* b = B + k * N;
+            for (int64_t j = 0; j < N; ++j) c[j] += a * (int64_t)b[j];
+        }
+    }
+}

@@ -200,6 +200,167 @@ encode_kxr_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
     }
 }
 
+// ---- 16-bit elements (12 significant bits): the table has 4096 entries of 64 bits (32 KB of shared
+// memory, one copy), indexed by the low 12 bits of the element.
+constexpr size_t kLut16SmemBytes = 4096 * sizeof(uint64_t);
+
+__device__ __forceinline__ uint2 lookup16(const unsigned char* lut_s, uint32_t byte_offset) {
+    return *reinterpret_cast<const uint2*>(lut_s + byte_offset);
+}
+
+// 8 elements held as 4 words (two 16-bit elements per word, ascending k) -> one output word per plane.
+template <int NP>
+__device__ __forceinline__ void encode8_16(const unsigned char* lut_s, const uint32_t (&w)[4], uint32_t (&out)[NP]) {
+    uint32_t lo[4], hi[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint2 e0 = lookup16(lut_s, (w[i] << 3) & 0x7FF8u);   // even k: bits 0-11 of the word
+        const uint2 e1 = lookup16(lut_s, (w[i] >> 13) & 0x7FF8u);  // odd k: bits 16-27
+        lo[i] = (e1.x << 4) + e0.x;
+        hi[i] = (e1.y << 4) + e0.y;
+    }
+    const uint32_t t01 = __byte_perm(lo[0], lo[1], 0x5140), t23 = __byte_perm(lo[2], lo[3], 0x5140);
+    out[0] = __byte_perm(t01, t23, 0x5410);
+    if (NP > 1) out[1 % NP] = __byte_perm(t01, t23, 0x7632);
+    if (NP > 2) {
+        const uint32_t u01 = __byte_perm(lo[0], lo[1], 0x7362), u23 = __byte_perm(lo[2], lo[3], 0x7362);
+        out[2 % NP] = __byte_perm(u01, u23, 0x5410);
+        if (NP > 3) out[3 % NP] = __byte_perm(u01, u23, 0x7632);
+    }
+    if (NP > 4) {
+        const uint32_t s01 = __byte_perm(hi[0], hi[1], 0x5140), s23 = __byte_perm(hi[2], hi[3], 0x5140);
+        out[4 % NP] = __byte_perm(s01, s23, 0x5410);
+        if (NP > 5) out[5 % NP] = __byte_perm(s01, s23, 0x7632);
+        if (NP > 6) {
+            const uint32_t v01 = __byte_perm(hi[0], hi[1], 0x7362), v23 = __byte_perm(hi[2], hi[3], 0x7362);
+            out[6 % NP] = __byte_perm(v01, v23, 0x5410);
+            if (NP > 7) out[7 % NP] = __byte_perm(v01, v23, 0x7632);
+        }
+    }
+}
+
+// 32 consecutive 16-bit elements of one plane row (16 words) -> 16 packed bytes per plane.
+template <int NP>
+__device__ __forceinline__ void encode32_16_store(const unsigned char* lut_s, const uint32_t (&in)[16], uint8_t* dst,
+                                                  int64_t plane_stride) {
+    uint32_t o[4][NP];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const uint32_t w[4] = {in[4 * g], in[4 * g + 1], in[4 * g + 2], in[4 * g + 3]};
+        encode8_16<NP>(lut_s, w, o[g]);
+    }
+#pragma unroll
+    for (int j = 0; j < NP; ++j)
+        *reinterpret_cast<uint4*>(dst + j * plane_stride) = make_uint4(o[0][j], o[1][j], o[2][j], o[3][j]);
+}
+
+__device__ __forceinline__ void load_lut16(unsigned char* lut_s, const uint64_t* __restrict__ lut_g) {
+    uint64_t* d = reinterpret_cast<uint64_t*>(lut_s);
+    for (int i = threadIdx.x; i < 4096; i += blockDim.x) d[i] = lut_g[i];
+    __syncthreads();
+}
+
+// 16-bit operand with the reduction index contiguous: a warp handles 1024 consecutive k of one row.
+template <int NP>
+__global__ void __launch_bounds__(kEncThreads)
+encode16_rxk_kernel(const uint16_t* __restrict__ X, int64_t R, int64_t K, int64_t ld,
+                    const uint64_t* __restrict__ lut_g, uint8_t* __restrict__ planes, int64_t pitch,
+                    int64_t plane_stride, int vec_ok) {
+    extern __shared__ __align__(128) unsigned char lut_s[];
+    load_lut16(lut_s, lut_g);
+    const int lane = threadIdx.x & 31;
+    const int64_t Kp = pitch * 2;
+    const int64_t chunks = (Kp + 1023) / 1024;
+    const int64_t items = R * chunks;
+    const int64_t warps_total = (int64_t)gridDim.x * (kEncThreads / 32);
+    for (int64_t it = (int64_t)blockIdx.x * (kEncThreads / 32) + (threadIdx.x >> 5); it < items; it += warps_total) {
+        const int64_t row = it / chunks, k0 = (it % chunks) * 1024 + lane * 32;
+        if (k0 >= Kp) continue;
+        uint32_t in[16];
+        const uint16_t* src = X + row * ld + k0;
+        if (vec_ok && k0 + 32 <= K) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint4 a = __ldg(reinterpret_cast<const uint4*>(src) + q);
+                in[4 * q] = a.x; in[4 * q + 1] = a.y; in[4 * q + 2] = a.z; in[4 * q + 3] = a.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int64_t k = k0 + 2 * i;
+                const uint32_t e0 = (k < K) ? (uint32_t)src[2 * i] : 0u;
+                const uint32_t e1 = (k + 1 < K) ? (uint32_t)src[2 * i + 1] : 0u;
+                in[i] = e0 | (e1 << 16);
+            }
+        }
+        encode32_16_store<NP>(lut_s, in, planes + row * pitch + k0 / 2, plane_stride);
+    }
+}
+
+// 16-bit operand with the reduction index strided (K x N): a lane owns 2 consecutive r and 32 k;
+// 4 neighbouring lanes cover 128 consecutive k of the same rows, so stores fill whole sectors.
+template <int NP>
+__global__ void __launch_bounds__(kEncThreads)
+encode16_kxr_kernel(const uint16_t* __restrict__ X, int64_t R, int64_t K, int64_t ld,
+                    const uint64_t* __restrict__ lut_g, uint8_t* __restrict__ planes, int64_t pitch,
+                    int64_t plane_stride, int vec_ok) {
+    extern __shared__ __align__(128) unsigned char lut_s[];
+    load_lut16(lut_s, lut_g);
+    const int lane = threadIdx.x & 31;
+    const int64_t Kp = pitch * 2;
+    constexpr int kRows = (32 / kKxrLanesK) * 2;
+    const int64_t k_items = (Kp + kKxrK - 1) / kKxrK, r_items = (R + kRows - 1) / kRows;
+    const int64_t items = k_items * r_items;
+    const int64_t warps_total = (int64_t)gridDim.x * (kEncThreads / 32);
+    for (int64_t it = (int64_t)blockIdx.x * (kEncThreads / 32) + (threadIdx.x >> 5); it < items; it += warps_total) {
+        const int64_t r0 = (it % r_items) * kRows + (lane / kKxrLanesK) * 2;
+        const int64_t k0 = (it / r_items) * kKxrK + (lane % kKxrLanesK) * 32;
+        if (r0 >= R || k0 >= Kp) continue;
+        uint32_t raw[32];  // raw[i] = elements X[k0+i][r0], X[k0+i][r0+1]
+        if (vec_ok && r0 + 2 <= R && k0 + 32 <= K) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) raw[i] = __ldg(reinterpret_cast<const uint32_t*>(X + (k0 + i) * ld + r0));
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                uint32_t word = 0;
+                if (k0 + i < K) {
+                    word = (uint32_t)X[(k0 + i) * ld + r0];
+                    if (r0 + 1 < R) word |= (uint32_t)X[(k0 + i) * ld + r0 + 1] << 16;
+                }
+                raw[i] = word;
+            }
+        }
+        uint32_t t0[16], t1[16];  // rows r0 and r0+1: 32 consecutive k each, two per word
+#pragma unroll
+        for (int g = 0; g < 16; ++g) {
+            t0[g] = __byte_perm(raw[2 * g], raw[2 * g + 1], 0x5410);
+            t1[g] = __byte_perm(raw[2 * g], raw[2 * g + 1], 0x7632);
+        }
+        encode32_16_store<NP>(lut_s, t0, planes + r0 * pitch + k0 / 2, plane_stride);
+        if (r0 + 1 < R) encode32_16_store<NP>(lut_s, t1, planes + (r0 + 1) * pitch + k0 / 2, plane_stride);
+    }
+}
+
+template <int NP>
+cudaError_t launch16(awe_layout_t layout, const uint16_t* X, int64_t R, int64_t K, int64_t ld, const uint64_t* lut,
+                     uint8_t* planes, int64_t pitch, int64_t plane_stride, int vec_ok, int sm_count,
+                     cudaStream_t stream) {
+    const int64_t warps_per_block = kEncThreads / 32;
+    const int64_t items = layout == AWE_ROWMAJOR_RxK
+                              ? R * ((pitch * 2 + 1023) / 1024)
+                              : ((pitch * 2 + kKxrK - 1) / kKxrK) * ((R + (32 / kKxrLanesK) * 2 - 1) / ((32 / kKxrLanesK) * 2));
+    const int64_t blocks =
+        std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
+    if (layout == AWE_ROWMAJOR_RxK)
+        encode16_rxk_kernel<NP><<<(unsigned)blocks, kEncThreads, kLut16SmemBytes, stream>>>(X, R, K, ld, lut, planes, pitch,
+                                                                                           plane_stride, vec_ok);
+    else
+        encode16_kxr_kernel<NP><<<(unsigned)blocks, kEncThreads, kLut16SmemBytes, stream>>>(X, R, K, ld, lut, planes, pitch,
+                                                                                           plane_stride, vec_ok);
+    return cudaGetLastError();
+}
+
 template <int NP>
 cudaError_t launch(awe_layout_t layout, const int8_t* X, int64_t R, int64_t K, int64_t ld, const uint64_t* lut,
                    uint8_t* planes, int64_t pitch, int64_t plane_stride, int vec_ok, int sm_count,
@@ -229,7 +390,7 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
                                    void* planes_dev, void* stream) {
     if (!h || !X_dev || !planes_dev || R <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
     if (side != AWE_SIDE_A && side != AWE_SIDE_B) return AWE_ERR_INVALID_ARG;
-    if ((int)dt < 0 || (int)dt > 2) return AWE_ERR_INVALID_ARG;
+    if ((int)dt < 0 || (int)dt > 3) return AWE_ERR_INVALID_ARG;
     if (layout != AWE_ROWMAJOR_RxK && layout != AWE_ROWMAJOR_KxR) return AWE_ERR_INVALID_ARG;
     if (ld < (layout == AWE_ROWMAJOR_RxK ? K : R)) return AWE_ERR_INVALID_ARG;
     if ((uintptr_t)planes_dev % 256) return AWE_ERR_ALIGNMENT;
@@ -243,9 +404,19 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
     // vector path: 16-byte loads along k (RxK) or 4-byte loads along r (KxR)
     const int64_t align = layout == AWE_ROWMAJOR_RxK ? 16 : 4;
     const int vec_ok = ((uintptr_t)X_dev % align == 0) && (ld % align == 0);
-    const int8_t* X = (const int8_t*)X_dev;
     uint8_t* P = (uint8_t*)planes_dev;
     cudaError_t e;
+    if (dt == AWE_I16) {
+        if ((uintptr_t)X_dev % 2) return AWE_ERR_ALIGNMENT;
+        const int vec16 = layout == AWE_ROWMAJOR_RxK ? (((uintptr_t)X_dev % 16 == 0) && (ld % 8 == 0))
+                                                     : (((uintptr_t)X_dev % 4 == 0) && (ld % 2 == 0));
+        if (t->n_planes != 6) return AWE_ERR_UNSUPPORTED;
+        e = launch16<6>(layout, (const uint16_t*)X_dev, R, K, ld, lut, P, pitch, plane_stride, vec16, h->sm_count, st);
+        if (e != cudaSuccess) return AWE_ERR_CUDA;
+        h->launches += 1;
+        return AWE_OK;
+    }
+    const int8_t* X = (const int8_t*)X_dev;
     switch (t->n_planes) {
         case 1: e = launch<1>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st); break;
         case 2: e = launch<2>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st); break;

@@ -30,9 +30,10 @@ struct SideTable {
     int n_planes = 0;
     int planes[AWE_MAX_PLANES][kMaxLimbs] = {{0}};
     int index_of_product[AWE_MAX_PRODUCTS] = {0};
-    int c = 0;                         // largest |plane value| over the input range
-    int8_t value[256][AWE_MAX_PLANES]; // plane values for raw byte b (index b & 0xFF)
-    uint64_t lut[256];                 // E2M1 code of plane j in the low nibble of byte j
+    int c = 0;       // largest |plane value| over the input range
+    int entries = 0; // 256 (index: raw byte) or 4096 (index: low 12 bits of a 16-bit element)
+    std::vector<int8_t> value;  // entries x AWE_MAX_PLANES plane values
+    std::vector<uint64_t> lut;  // entries words: E2M1 code of plane j in the low nibble of byte j
 };
 
 // Builds (and caches) scheme + tables; returns false if the encoding/modulus is not available.
@@ -42,6 +43,7 @@ awe_in_dtype_t natural_dtype(int enc, awe_side_t side);
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 inline int64_t plane_pitch_bytes(int64_t K) { return round_up(K, 256) / 2; }
+inline int64_t in_elem_bytes(awe_in_dtype_t dt) { return dt == AWE_I16 ? 2 : 1; }
 
 }  // namespace awe
 
@@ -50,6 +52,11 @@ struct awe_ctx {
     int sm_count = 0;
     unsigned int* status_dev = nullptr;  // [0] = status, [1] = site, [2..5] = clock probe of the last GEMM launch
     uint64_t* lut_arena_dev = nullptr;   // kLutSlots tables of 256 x u64
+    uint64_t* lut16_arena_dev = nullptr; // kLut16Slots tables of 4096 x u64 (16-bit inputs)
+    struct Lut16Slot {
+        int enc, side;
+    };
+    std::vector<Lut16Slot> slots16;
     struct LutSlot {
         int enc, modulus, side, dt;
     };
@@ -67,6 +74,7 @@ struct awe_ctx {
 
 namespace awe {
 constexpr int kLutSlots = 96;
+constexpr int kLut16Slots = 4;
 constexpr int kStatusWords = 8;
 // Device pointer of the 256-entry u64 table for (enc, modulus, side, dt); uploads on first use.
 awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_in_dtype_t dt,

@@ -120,6 +120,38 @@ Scheme make_int4x4() {
     return s;
 }
 
+Scheme make_fp16sig() {
+    // A = a0 + 9 a1 + 71 a2 + 639 a3 (same for B); with P_ij = a_i b_j and
+    // Q_kl = (a_2k + 2 a_2k+1)(b_2l + 2 b_2l+1):
+    //   2AB = sum_{k,l} 71^(k+l) (-7 P[2k,2l] + 126 P[2k+1,2l+1] + 9 Q[k,l])        (Appendix A)
+    Scheme s;
+    s.p = s.q = 4;
+    s.r = 12;
+    set_vec(s.w, {1, 9, 71, 639});
+    set_vec(s.v, {1, 9, 71, 639});
+    const int pw[3] = {1, 71, 5041};
+    int n = 0;
+    for (int k = 0; k < 2; ++k)
+        for (int l = 0; l < 2; ++l) {
+            const int sc = pw[k + l];
+            s.alpha[n][2 * k] = 1;
+            s.beta[n][2 * l] = 1;
+            s.ell[n++] = -7 * sc;
+            s.alpha[n][2 * k + 1] = 1;
+            s.beta[n][2 * l + 1] = 1;
+            s.ell[n++] = 126 * sc;
+            s.alpha[n][2 * k] = 1;
+            s.alpha[n][2 * k + 1] = 2;
+            s.beta[n][2 * l] = 1;
+            s.beta[n][2 * l + 1] = 2;
+            s.ell[n++] = 9 * sc;
+        }
+    s.log2D = 1;
+    s.a_lo = s.b_lo = -2048;
+    s.a_hi = s.b_hi = 2047;
+    return s;
+}
+
 struct Choice {
     int max_abs, sum_abs;
     int limbs[kMaxLimbs];
@@ -279,6 +311,7 @@ std::map<std::tuple<int, int, int, int>, SideTable> g_tables;
 awe_in_dtype_t natural_dtype(int enc, awe_side_t side) {
     if (enc == AWE_ENC_INT4xINT8_AWE4 && side == AWE_SIDE_A) return AWE_I4_IN_I8;
     if (enc == AWE_ENC_INT4xINT4_3) return AWE_I4_IN_I8;
+    if (enc == AWE_ENC_FP16SIG_AWE12) return AWE_I16;
     if (enc == AWE_ENC_TERNARY_INT8_3 && side == AWE_SIDE_A) return AWE_T2_IN_I8;
     return AWE_I8;
 }
@@ -309,6 +342,10 @@ bool get_scheme(int enc, int modulus, Scheme* out) {
             break;
         case AWE_ENC_INT4xINT8_AWE4:
             s = make_awe4();
+            ok = true;
+            break;
+        case AWE_ENC_FP16SIG_AWE12:
+            s = make_fp16sig();
             ok = true;
             break;
         case AWE_ENC_INT4xINT4_3:
@@ -342,8 +379,9 @@ bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, co
         return true;
     }
     SideTable t;
-    memset(t.value, 0, sizeof(t.value));
-    memset(t.lut, 0, sizeof(t.lut));
+    t.entries = dt == AWE_I16 ? 4096 : 256;
+    t.value.assign((size_t)t.entries * AWE_MAX_PLANES, 0);
+    t.lut.assign((size_t)t.entries, 0);
     stored_planes(s, side, &t);
     const int n = side == AWE_SIDE_A ? s.p : s.q;
     const int* weights = side == AWE_SIDE_A ? s.w : s.v;
@@ -352,10 +390,11 @@ bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, co
     const int lo = side == AWE_SIDE_A ? s.a_lo : s.b_lo;
     const int hi = side == AWE_SIDE_A ? s.a_hi : s.b_hi;
     t.c = 0;
-    for (int b = 0; b < 256; ++b) {
+    for (int b = 0; b < t.entries; ++b) {
         int x = (int)(int8_t)b;
         if (dt == AWE_I4_IN_I8) x = (int)(int8_t)((b & 0xF) << 4) >> 4;  // low nibble, sign-extended
         if (dt == AWE_T2_IN_I8 && (x < -1 || x > 1)) x = 0;              // not a ternary value
+        if (dt == AWE_I16) x = (int)(int16_t)((b & 0xFFF) << 4) >> 4;     // low 12 bits, sign-extended
         int key_x = x;
         if (s.modulus) {
             key_x = ((x % s.modulus) + s.modulus) % s.modulus;
@@ -368,7 +407,7 @@ bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, co
         for (int j = 0; j < t.n_planes; ++j) {
             int pv = 0;
             for (int i = 0; i < n; ++i) pv += t.planes[j][i] * f->second.limbs[i];
-            t.value[b][j] = (int8_t)pv;
+            t.value[(size_t)b * AWE_MAX_PLANES + j] = (int8_t)pv;
             t.c = std::max(t.c, std::abs(pv));
             word |= (uint64_t)e2m1_code_of(pv) << (8 * j);
         }
@@ -414,12 +453,12 @@ extern "C" awe_status_t awe_encoding_info(int enc, int modulus, awe_encoding_des
 
 extern "C" awe_status_t awe_encoding_lut(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt,
                                          int8_t* lut_host) {
-    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (int)dt < 0 || (int)dt > 2)
+    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (int)dt < 0 || (int)dt > 3)
         return AWE_ERR_INVALID_ARG;
     const SideTable* t;
     if (!get_side_table(enc, modulus, side, dt, &t)) return AWE_ERR_UNSUPPORTED;
-    for (int b = 0; b < 256; ++b)
-        for (int j = 0; j < t->n_planes; ++j) lut_host[b * t->n_planes + j] = t->value[b][j];
+    for (int b = 0; b < t->entries; ++b)
+        for (int j = 0; j < t->n_planes; ++j) lut_host[b * t->n_planes + j] = t->value[(size_t)b * AWE_MAX_PLANES + j];
     return AWE_OK;
 }
 

@@ -35,7 +35,7 @@ def gpu_encode(enc, modulus, side, X_rk, dt=b.I8, layout=b.ROWMAJOR_RxK, ld_extr
     src = X_rk if layout == b.ROWMAJOR_RxK else np.ascontiguousarray(X_rk.T)
     rows, cols = src.shape
     ld = cols + ld_extra
-    buf = np.zeros(rows * ld + offset, dtype=np.int8)
+    buf = np.zeros(rows * ld + offset, dtype=X_rk.dtype)
     view = buf[offset:offset + rows * ld].reshape(rows, ld)
     view[:, :cols] = src
     dX = torch.from_numpy(buf).cuda()

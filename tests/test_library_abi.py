@@ -41,6 +41,13 @@ def test_records_match_the_paper_and_the_oracle(b):
     s = sc.TERNARY3
     assert d.r == 3 and list(d.ell)[:3] == list(s.ell) and list(d.ib)[:3] == s.plane_index("B")
     assert (d.n_planes_a, d.n_planes_b, d.c_a, d.c_b, d.k_star) == (1, 3, 1, 8, 2097152)
+    d = b.awe_encoding_info(b.ENC_FP16SIG_AWE12)
+    s = sc.FP16_M12
+    assert d.r == 12 and list(d.ell)[:12] == list(s.ell) and d.log2D == 1
+    assert list(d.ia)[:12] == s.plane_index("A") and list(d.ib)[:12] == s.plane_index("B")
+    assert (d.n_planes_a, d.n_planes_b, d.c_a, d.c_b, d.k_star) == (6, 6, 12, 12, 116508)
+    lut = b.awe_encoding_lut(b.ENC_FP16SIG_AWE12, 0, b.SIDE_A, b.I16)
+    assert np.array_equal(lut[np.arange(-2047, 2048) & 0xFFF], pl.plane_lut(sc.FP16_M12, "A", -2047, 2047))
     d = b.awe_encoding_info(b.ENC_INT4xINT4_3)
     assert d.r == 3 and list(d.ell)[:3] == list(sc.INT4X4_3.ell) and (d.c_a, d.c_b, d.k_star) == (2, 2, 4194304)
     lut = b.awe_encoding_lut(b.ENC_INT4xINT4_3, 0, b.SIDE_B, b.I4_IN_I8)

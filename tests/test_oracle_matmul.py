@@ -45,6 +45,17 @@ def test_closed_forms():
     assert mm.matmul_i64(A, Bm).tolist() == [[2, 3], [4, 7]]
 
 
+def test_int16_product_against_numpy_and_python():
+    rng = np.random.default_rng(12)
+    A = rng.integers(-2047, 2048, (9, 33), dtype=np.int16)
+    B = rng.integers(-2047, 2048, (33, 7), dtype=np.int16)
+    C = mm.matmul_i64_s16(A, B)
+    assert np.array_equal(C, A.astype(np.int64) @ B.astype(np.int64))
+    assert np.array_equal(C, _py_matmul(A, B))
+    assert np.array_equal(mm.matmul_i64_s16(A, B, 2, 5), C[2:5])
+    assert np.array_equal(pl.awe_matmul(sc.FP16_M12, A, B, a_range=(-2047, 2047), b_range=(-2047, 2047)), C)
+
+
 def test_mod_symmetric():
     C = np.arange(-50, 50, dtype=np.int64).reshape(10, 10)
     for m in (7, 8, 13):
