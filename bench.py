@@ -294,7 +294,7 @@ def main():
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
                      "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_BYTES_8192 if (M, N, K) == (8192, 8192, 8192) else None,
                      "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one launch at this workload "
-                                     "(ncu, one-pass metrics; profiles/launch_list_bench_8192_awe6.md)",
+                                     "(ncu capture with one-pass metrics; summary kept under profiles/)",
                      "kernel": "awe_gemm_kernel", "flops_per_launch": desc.r * ops,
                      "peak_source": "%s bf16 sustained %.1f TFLOP/s x nominal fp4:bf16 ratio 4" %
                                     (peaks["source"], peaks["bf16_tflops_sustained"]),
@@ -306,6 +306,23 @@ def main():
                             "peak": peaks["hbm_gbs"], "unit": "GB/s"},
     }
     line["encode_roofline"]["frac"] = line["encode_roofline"]["achieved"] / peaks["hbm_gbs"]
+    # The encode writes 3 bytes for every byte it reads, and HBM writes alone run well below the
+    # read+write copy figure: measure a plain fill of the same size and report the write stream against it.
+    fill_buf = torch.empty(int((M * K + K * N) * desc.n_planes_a / 2), dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        fill_buf.fill_(1)
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    f0.record()
+    for _ in range(10):
+        fill_buf.fill_(1)
+    f1.record()
+    torch.cuda.synchronize()
+    fill_gbs = fill_buf.numel() / (f0.elapsed_time(f1) / 10 * 1e-3) / 1e9
+    enc_write_gbs = fill_buf.numel() / (ms_encode * 1e-3) / 1e9
+    line["encode_roofline"].update({"write_GBs": enc_write_gbs, "fill_GBs_measured_now": fill_gbs,
+                                    "frac_of_write_bandwidth": enc_write_gbs / fill_gbs})
+    del fill_buf
 
     if rank == 0 and not args.no_extras:
         ctx = {}

@@ -7,8 +7,10 @@
 // with one shift-add per 32-bit half (the odd element moves to the high nibbles), which yields
 // the packed output byte of every plane at once; byte permutes then gather 4 such words into one
 // 32-bit output word per plane.  In shared memory every table entry is 128 bytes wide and holds
-// one copy per lane (16 copies of the 64-bit word, or 32 copies of its low half when there are at
-// most 4 planes), so a warp's data-dependent lookups never collide on a bank.
+// one 32-bit copy per lane, so a warp's data-dependent lookups never collide on a bank and cost
+// one shared-memory wavefront each.  With 5 or 6 planes the codes of planes 4 and 5 ride in the
+// (otherwise empty) high nibbles of bytes 0 and 1 of that word; with 7 or 8 planes the entry is the
+// full 64-bit word, 16 copies.
 #include <algorithm>
 
 #include "awe_internal.h"
@@ -30,12 +32,16 @@ constexpr int kKxrK = kKxrLanesK * 32;                // k per warp item
 
 template <int NP>
 __device__ __forceinline__ void load_lut(unsigned char* lut_s, const uint64_t* __restrict__ lut_g) {
-    if (NP > 4) {
+    if (NP > 6) {
         uint64_t* d = reinterpret_cast<uint64_t*>(lut_s);
         for (int i = threadIdx.x; i < 256 * 16; i += blockDim.x) d[i] = lut_g[i >> 4];
     } else {
         uint32_t* d = reinterpret_cast<uint32_t*>(lut_s);
-        for (int i = threadIdx.x; i < 256 * 32; i += blockDim.x) d[i] = (uint32_t)lut_g[i >> 5];
+        for (int i = threadIdx.x; i < 256 * 32; i += blockDim.x) {
+            const uint64_t e = lut_g[i >> 5];
+            // planes 0-3 stay in the low nibbles of bytes 0-3; planes 4, 5 move to the high nibbles of bytes 0, 1
+            d[i] = (uint32_t)e | (((uint32_t)(e >> 32) & 0x0F0Fu) << 4);
+        }
     }
     __syncthreads();
 }
@@ -43,7 +49,7 @@ __device__ __forceinline__ void load_lut(unsigned char* lut_s, const uint64_t* _
 // Byte offset of this lane's private copy inside a 128-byte table entry.
 template <int NP>
 __device__ __forceinline__ uint32_t lane_slot(int lane) {
-    return NP > 4 ? (uint32_t)(lane & 15) * 8u : (uint32_t)lane * 4u;
+    return NP > 6 ? (uint32_t)(lane & 15) * 8u : (uint32_t)lane * 4u;
 }
 
 // Table words (low half: planes 0-3, high half: planes 4-7) of byte number I of `word`.
@@ -52,7 +58,7 @@ __device__ __forceinline__ uint2 lookup(const unsigned char* lut_s, uint32_t slo
     // entry address = byte * 128; the lane slot occupies bits below 7 and is OR-ed in
     const uint32_t shifted = I == 0 ? (word << 7) : (word >> (8 * I - 7));
     const uint32_t off = (shifted & 0x7F80u) | slot;
-    if (NP > 4) return *reinterpret_cast<const uint2*>(lut_s + off);
+    if (NP > 6) return *reinterpret_cast<const uint2*>(lut_s + off);
     return make_uint2(*reinterpret_cast<const uint32_t*>(lut_s + off), 0u);
 }
 
@@ -65,8 +71,20 @@ __device__ __forceinline__ void encode8(const unsigned char* lut_s, uint32_t slo
     const uint2 e4 = lookup<NP, 0>(lut_s, slot, w1), e5 = lookup<NP, 1>(lut_s, slot, w1);
     const uint2 e6 = lookup<NP, 2>(lut_s, slot, w1), e7 = lookup<NP, 3>(lut_s, slot, w1);
     // pair words: byte j = packed byte (even k low nibble, odd k high nibble) of plane j
-    const uint32_t l0 = (e1.x << 4) + e0.x, l1 = (e3.x << 4) + e2.x, l2 = (e5.x << 4) + e4.x,
-                   l3 = (e7.x << 4) + e6.x;
+    uint32_t l0, l1, l2, l3, h0 = 0, h1 = 0, h2 = 0, h3 = 0;
+    if (NP <= 4) {
+        l0 = (e1.x << 4) + e0.x; l1 = (e3.x << 4) + e2.x; l2 = (e5.x << 4) + e4.x; l3 = (e7.x << 4) + e6.x;
+    } else if (NP <= 6) {
+        // compact entries: low nibbles = planes 0-3, high nibbles of bytes 0, 1 = planes 4, 5
+        const uint32_t m = 0x0F0F0F0Fu;
+        l0 = (e0.x & m) | ((e1.x << 4) & ~m); l1 = (e2.x & m) | ((e3.x << 4) & ~m);
+        l2 = (e4.x & m) | ((e5.x << 4) & ~m); l3 = (e6.x & m) | ((e7.x << 4) & ~m);
+        h0 = ((e0.x >> 4) & 0x0F0Fu) | (e1.x & 0xF0F0u); h1 = ((e2.x >> 4) & 0x0F0Fu) | (e3.x & 0xF0F0u);
+        h2 = ((e4.x >> 4) & 0x0F0Fu) | (e5.x & 0xF0F0u); h3 = ((e6.x >> 4) & 0x0F0Fu) | (e7.x & 0xF0F0u);
+    } else {
+        l0 = (e1.x << 4) + e0.x; l1 = (e3.x << 4) + e2.x; l2 = (e5.x << 4) + e4.x; l3 = (e7.x << 4) + e6.x;
+        h0 = (e1.y << 4) + e0.y; h1 = (e3.y << 4) + e2.y; h2 = (e5.y << 4) + e4.y; h3 = (e7.y << 4) + e6.y;
+    }
     const uint32_t t01 = __byte_perm(l0, l1, 0x5140), t23 = __byte_perm(l2, l3, 0x5140);
     out[0] = __byte_perm(t01, t23, 0x5410);
     if (NP > 1) out[1 % NP] = __byte_perm(t01, t23, 0x7632);
@@ -76,8 +94,6 @@ __device__ __forceinline__ void encode8(const unsigned char* lut_s, uint32_t slo
         if (NP > 3) out[3 % NP] = __byte_perm(u01, u23, 0x7632);
     }
     if (NP > 4) {
-        const uint32_t h0 = (e1.y << 4) + e0.y, h1 = (e3.y << 4) + e2.y, h2 = (e5.y << 4) + e4.y,
-                       h3 = (e7.y << 4) + e6.y;
         const uint32_t s01 = __byte_perm(h0, h1, 0x5140), s23 = __byte_perm(h2, h3, 0x5140);
         out[4 % NP] = __byte_perm(s01, s23, 0x5410);
         if (NP > 5) out[5 % NP] = __byte_perm(s01, s23, 0x7632);
