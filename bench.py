@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 METRIC = "effective exact INT8xINT8 TOPS (2*M*N*K / time), AWE 6-GEMM"
 NOMINAL_FP4_TFLOPS = 9000.0          # published dense FP4 peak of one B200 (paper, Section 6.2)
 NOMINAL_FP4_OVER_BF16 = 4.0          # 9.0 / 2.25 PFLOP/s nominal
-GEMM_DRAM_BYTES_8192 = 1524829696 + 262142208   # ncu capture of awe_gemm_kernel at 8192^3, AWE-6
+GEMM_DRAM_BYTES_8192 = 1646774784 + 356711424   # ncu capture of awe_gemm_kernel at 8192^3, AWE-6
 MAC_PER_CLK_PER_SM = 16384           # dense FP4: 4 x the 4096 bf16 MAC/clk/SM of the tcgen05 pipe
 
 
