@@ -223,7 +223,8 @@ awe_status_t awe_gemm_exact_wide(awe_handle_t h, const int64_t* A_dev, const int
  *   - A_dev, B_dev, C_dev, dtypes, sizes, enc, modulus, out_dt: exactly as for awe_gemm_exact
  *     (A: M x K, B: K x N, C: M x N, all row-major and dense).
  *   - AWE_ERR_WORKSPACE if awe_workspace_bytes(enc, modulus, M, N, K) exceeds
- *     AWE_STATIC_WORKSPACE_BYTES; nothing is enqueued then.
+ *     AWE_STATIC_WORKSPACE_BYTES; nothing is enqueued then.  Encodings with 16-bit inputs are not
+ *     served (AWE_ERR_UNSUPPORTED): their 32 KB tables have no room in the built-in array.
  *   - The first call on a device looks up the array's device address and the device's properties
  *     and clears the status word; the first use of an encoding on a device uploads its tables and
  *     waits for that copy.  Make those first calls before any stream capture.

@@ -50,7 +50,7 @@ struct Cfg {
     static constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | (1u << 23) |
                                        ((uint32_t)((kTileM * kCtas) >> 4) << 24);
 };
-constexpr int kMaxStages = 7;
+constexpr int kMaxStages = 6;
 // Two accumulators of 256 columns and 32 columns of scale bytes do not fit 512 columns side by
 // side, so accumulator 1 starts inside the last 32 columns of accumulator 0.  The epilogue reads
 // those shared columns first and releases them separately (overlap_free), which lets the MMAs of

@@ -132,6 +132,25 @@ def test_residue_form_every_modulus_of_the_set(m):
     assert np.array_equal(gu.gpu_gemm_exact(A, B, b.ENC_MOD_M, b.C_RES_I32, modulus=m), want)
 
 
+@pytest.mark.parametrize("m,K,k_chunk", [(157, 49152, 256), (89, 8192, 512), (13, 4096, 256)])
+def test_residue_form_with_many_k_segments(m, K, k_chunk):
+    """Many exact-accumulation segments per product: the running residue sum must be reduced on
+    the way (for m = 157 and 192 segments it would otherwise leave the exact float range)."""
+    w = wl.small("t", 128, 256, K, "residue", "residue", seed=m, modulus=m)
+    A, B = wl.make_inputs(w)
+    want = mm.mod_symmetric(mm.matmul_i64(A, B), m)
+    pa = gu.gpu_encode(b.ENC_MOD_M, m, b.SIDE_A, A)
+    pb = gu.gpu_encode(b.ENC_MOD_M, m, b.SIDE_B, np.ascontiguousarray(B.T))
+    got = gu.gpu_gemm_planes(pa, pb, w.M, w.N, w.K, b.ENC_MOD_M, b.C_RES_I16, modulus=m, k_chunk=k_chunk)
+    assert np.array_equal(got, want)
+
+
+def test_tall_and_wide_shapes():
+    for (M, N, K) in [(5000, 64, 320), (64, 5000, 320), (3, 1030, 7), (1030, 3, 7)]:
+        A, B = wl.make_inputs(wl.small("t", M, N, K, seed=M + N))
+        assert np.array_equal(gu.gpu_gemm_exact(A, B, b.ENC_INT8_AWE6, b.C_I32), mm.matmul_i64(A, B))
+
+
 def test_residue_form_accepts_any_int8_input():
     A, B = wl.make_inputs(wl.small("t", 128, 256, 512, seed=4))
     want = mm.mod_symmetric(mm.matmul_i64(A, B), 61)
