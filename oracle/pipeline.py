@@ -11,6 +11,7 @@ produced only by pack_e2m1, which mirrors what the hardware stores (Section 3.1)
 """
 from __future__ import annotations
 
+import functools
 from typing import Dict, List, Optional, Sequence, Tuple
 
 import numpy as np
@@ -19,8 +20,10 @@ from .schemes import (F_ACC, S_SET, Scheme, dot, e2m1_code, k_star, symmetric_ra
                       to_symmetric, value_table)
 
 
+@functools.lru_cache(maxsize=None)
 def encoder_table(s: Scheme, side: str) -> Dict[int, Tuple[int, ...]]:
-    """Decomposition table of one side of a scheme (first loop of Algorithm 1)."""
+    """Decomposition table of one side of a scheme (first loop of Algorithm 1).  Built once per
+    (scheme, side): the table is a constant of the configuration record."""
     weights, planes = s.side(side)
     return value_table(weights, planes, modulus=s.modulus)
 
@@ -33,6 +36,7 @@ def plane_values(s: Scheme, side: str, x: int) -> List[int]:
     return [dot(p, a) for p in s.stored_planes(side)]
 
 
+@functools.lru_cache(maxsize=None)
 def plane_lut(s: Scheme, side: str, lo: int, hi: int) -> np.ndarray:
     """(hi-lo+1) x n_planes int8 array of stored plane values for inputs lo..hi."""
     t = encoder_table(s, side)

@@ -86,6 +86,19 @@ def test_algorithm1_residue_form(m):
     assert np.array_equal(pl.awe_matmul(sc.mod_scheme(m), A, B), want)
 
 
+def test_brute_force_all_2x2x2_matrices_over_extreme_values():
+    """Every 2x2 by 2x2 product with entries from {-128, 0, 127}: Algorithm 1 (6-product and
+    base-13 encodings) against integer arithmetic written out entry by entry."""
+    import itertools
+    vals = (-128, 0, 127)
+    mats = [np.array(c, dtype=np.int8).reshape(2, 2) for c in itertools.product(vals, repeat=4)]
+    for s in (sc.AWE6, sc.BASE13_9):
+        for A in mats:
+            for B in mats[::3]:
+                want = [[int(A[i, 0]) * int(B[0, j]) + int(A[i, 1]) * int(B[1, j]) for j in range(2)] for i in range(2)]
+                assert pl.awe_matmul(s, A, B).tolist() == want
+
+
 def test_config1_all_int8_encodings_agree():
     A, B = wl.make_inputs(wl.config1())
     C = mm.matmul_i64(A, B)
