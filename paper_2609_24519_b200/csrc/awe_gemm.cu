@@ -454,7 +454,7 @@ template <bool kPair>
 awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p,
                             cudaStream_t st) {
     using C = Cfg<kPair>;
-    static bool attr_set = false;
+    bool& attr_set = h->smem_attr_set[kPair ? 0 : 1];
     if (!attr_set) {
         if (cudaFuncSetAttribute(awe_gemm_kernel<kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)C::kSmemBytes) != cudaSuccess)

@@ -234,7 +234,7 @@ namespace gemm {
 int wide_b_box_rows() { return kBRows; }
 
 awe_status_t launch_gemm_wide(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
-    static bool attr_set = false;
+    bool& attr_set = h->smem_attr_set[2];
     if (!attr_set) {
         if (cudaFuncSetAttribute(awe_gemm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) !=
             cudaSuccess)

@@ -69,7 +69,7 @@ struct awe_ctx {
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_done = nullptr;
     cudaEvent_t ev_a[kMaxHostChunks] = {nullptr}, ev_c[kMaxHostChunks] = {nullptr};
-    std::mutex mu;
+    bool smem_attr_set[3] = {false, false, false};  // dynamic shared-memory limit raised (per kernel, this device)
 };
 
 namespace awe {

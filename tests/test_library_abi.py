@@ -88,3 +88,12 @@ def test_sizes_and_host_side_rejections(b):
     with pytest.raises(b.AweError):
         b.awe_encoding_info(b.ENC_INT8_AWE6, 7)
     assert "workspace" in b.status_string(3)
+
+
+def test_header_is_plain_c():
+    """include/awe.h must compile as C (no C++ in the boundary)."""
+    import subprocess
+    src = '#include "awe.h"\nint main(void) { awe_encoding_desc d; (void)d; return (int)AWE_OK; }\n'
+    r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-fsyntax-only", "-I", os.path.join(ROOT, "include"),
+                        "-x", "c", "-"], input=src, capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
