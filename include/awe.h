@@ -25,6 +25,9 @@
  *     device can see (a bounded wait inside a kernel ran out) are recorded in the handle's
  *     status word and reported by awe_last_device_status.
  *   - There is no CPU fallback: without a CUDA device awe_create fails with AWE_ERR_CUDA.
+ *   - The first use of an encoding on a handle uploads its tables and waits for that copy; from then
+ *     on awe_encode, awe_gemm_planes and awe_gemm_exact only enqueue kernels on `stream`, so a
+ *     warmed-up call can be captured in a CUDA graph and replayed (the tests do this).
  *   - One handle serves one device; calls on one handle must not run concurrently from
  *     several host threads.
  */

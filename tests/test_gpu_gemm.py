@@ -316,3 +316,29 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
     assert b.awe_last_device_status(h) == (0, 0)
     assert np.array_equal(C.cpu().numpy(), mm.matmul_i64(A, B))
     b.awe_destroy(h)
+
+
+def test_whole_procedure_can_be_captured_in_a_cuda_graph_and_replayed():
+    """After the first call (which uploads the tables) awe_gemm_exact only enqueues kernels, so a
+    launch-bound small product can be captured once and replayed."""
+    h = gu.handle()
+    w = wl.config1()
+    A, B = wl.make_inputs(w)
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    ws = torch.empty(b.awe_workspace_bytes(b.ENC_INT8_AWE6, 0, w.M, w.N, w.K), dtype=torch.uint8, device="cuda")
+    C = torch.zeros((w.M, w.N), dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, w.M, w.N, w.K, b.ENC_INT8_AWE6, 0, C, b.C_I32, ws)   # warm-up
+    side.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, w.M, w.N, w.K, b.ENC_INT8_AWE6, 0, C, b.C_I32, ws)
+    want = mm.matmul_i64(A, B)
+    for rep in range(3):
+        dA.copy_(torch.from_numpy(np.roll(A, rep, axis=0)).cuda())       # new data, same buffers
+        C.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(C.cpu().numpy(), np.roll(want, rep, axis=0))
+    assert b.awe_last_device_status(h) == (0, 0)
