@@ -181,11 +181,19 @@ awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, awe_in_dtyp
  * The inputs are split into symmetric residues modulo pairwise coprime moduli, each residue product
  * runs as a mod-m product on the FP4 kernels, and the Chinese remainder theorem rebuilds the exact
  * integers.  The built-in set has 22 moduli (60 FP4 GEMMs) with product 2^122.86, which gives a
- * unique result whenever 2 K (2^(in_bits-1) - 1)^2 stays below it: in_bits = 54 up to K = 59,000. */
+ * unique result whenever 2 K (2^(in_bits-1) - 1)^2 stays below it: in_bits = 54 up to K = 59,000.
+ * Narrower inputs use a cheaper subset (awe_wide_select). */
 
 /* The moduli of the built-in set: writes up to `capacity` of them to out (may be NULL), returns
  * how many there are.  Host only. */
 int awe_wide_moduli(int32_t* out, int capacity);
+
+/* The subset of the built-in moduli awe_gemm_exact_wide uses for inputs of `in_bits` bits and
+ * reduction length K: the one with the fewest FP4 products whose product exceeds
+ * 2 K (2^(in_bits-1) - 1)^2 (the selection problem of Section 5.3, solved exactly over the built-in
+ * set).  Writes up to `capacity` moduli to out (may be NULL) and returns their number, 0 if even the
+ * whole set is too small.  Host only. */
+int awe_wide_select(int in_bits, int64_t K, int32_t* out, int capacity);
 
 /* Bytes of scratch awe_gemm_exact_wide needs: residues of A and B (int8, one copy per modulus),
  * the residue products (int16 per modulus) and the plane workspace of one modulus. */

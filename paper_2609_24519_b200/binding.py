@@ -31,7 +31,7 @@ STATIC_WORKSPACE_BYTES = 24 << 20
 
 EXPORTS = ["awe_create", "awe_destroy", "awe_encoding_info", "awe_encoding_lut", "awe_planes_bytes",
            "awe_workspace_bytes", "awe_host_staging_bytes", "awe_encode", "awe_gemm_planes", "awe_gemm_exact",
-           "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_wide_moduli", "awe_wide_workspace_bytes",
+           "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_wide_moduli", "awe_wide_select", "awe_wide_workspace_bytes",
            "awe_wide_residues", "awe_wide_crt", "awe_gemm_exact_wide", "awe_reconstruct", "awe_fp4_product_raw", "awe_last_device_status", "awe_selftest_bounded_wait", "awe_last_gemm_clock_mhz", "awe_launch_count",
            "awe_status_string"]
 
@@ -79,6 +79,7 @@ def lib() -> ctypes.CDLL:
     L.awe_gemm_exact_host.argtypes = [vp, vp, i32, vp, i32, i64, i64, i64, i32, i32, vp, i32, vp, sz, vp]
     L.awe_gemm_exact_static.argtypes = [vp, i32, vp, i32, i64, i64, i64, i32, i32, vp, i32, vp]
     L.awe_wide_moduli.argtypes = [vp, i32]
+    L.awe_wide_select.argtypes = [i32, i64, vp, i32]
     L.awe_wide_workspace_bytes.argtypes = [i64, i64, i64]
     L.awe_wide_workspace_bytes.restype = sz
     L.awe_wide_residues.argtypes = [vp, vp, i64, vp, vp]
@@ -228,6 +229,13 @@ def awe_wide_moduli():
     out = (ctypes.c_int32 * n)()
     lib().awe_wide_moduli(out, n)
     return list(out)
+
+
+def awe_wide_select(in_bits: int, K: int):
+    n = lib().awe_wide_select(in_bits, K, None, 0)
+    out = (ctypes.c_int32 * max(n, 1))()
+    lib().awe_wide_select(in_bits, K, out, n)
+    return list(out)[:n]
 
 
 def awe_wide_workspace_bytes(M: int, N: int, K: int) -> int:

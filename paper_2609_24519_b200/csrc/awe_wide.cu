@@ -146,12 +146,12 @@ wide_crt_kernel(const short* __restrict__ res, long long count, const __grid_con
     }
 }
 
-bool build_crt_params(CrtParams* c) {
-    c->n = kNumWideModuli;
+bool build_crt_params(const int* moduli, int n, CrtParams* c) {
+    c->n = n;
     u128 M = 1;
-    for (int t = 0; t < kNumWideModuli; ++t) M *= (u128)kWideModuli[t];
-    for (int t = 0; t < kNumWideModuli; ++t) {
-        const int m = kWideModuli[t];
+    for (int t = 0; t < n; ++t) M *= (u128)moduli[t];
+    for (int t = 0; t < n; ++t) {
+        const int m = moduli[t];
         const u128 Mt = M / (u128)m;
         const int mt_mod = (int)(Mt % (u128)m);
         int inv = 0;
@@ -171,10 +171,50 @@ bool build_crt_params(CrtParams* c) {
     return true;
 }
 
-long double log2_of_moduli_product() {
-    long double s = 0;
-    for (int t = 0; t < kNumWideModuli; ++t) s += log2l((long double)kWideModuli[t]);
-    return s;
+// Number of FP4 products the residue scheme of modulus m needs (1, 3 or 4).
+int products_of(int m) {
+    awe_encoding_desc d;
+    return awe_encoding_info(AWE_ENC_MOD_M, m, &d) == AWE_OK ? d.r : 1 << 20;
+}
+
+// The paper chooses, by an integer program over the per-modulus costs, the moduli with the fewest
+// products whose product exceeds 2 K B^2 (Section 5.3).  Over the 22 built-in moduli this is a small
+// knapsack: best[c] = largest sum of log2(m) reachable with exactly c products; the cheapest c that
+// reaches the bound wins and the exact inequality is re-checked in integers.
+int select_moduli(int in_bits, int64_t K, int* out) {
+    const long double need = 1.0L + log2l((long double)K) + 2.0L * (long double)(in_bits - 1);
+    constexpr int kMaxCost = 64;
+    long double best[kMaxCost + 1];
+    unsigned int pick[kMaxCost + 1];
+    for (int c = 0; c <= kMaxCost; ++c) {
+        best[c] = -1;
+        pick[c] = 0;
+    }
+    best[0] = 0;
+    for (int t = 0; t < kNumWideModuli; ++t) {
+        const int cost = products_of(kWideModuli[t]);
+        const long double lg = log2l((long double)kWideModuli[t]);
+        for (int c = kMaxCost; c >= cost; --c)
+            if (best[c - cost] >= 0 && best[c - cost] + lg > best[c]) {
+                best[c] = best[c - cost] + lg;
+                pick[c] = pick[c - cost] | (1u << t);
+            }
+    }
+    for (int c = 1; c <= kMaxCost; ++c) {
+        if (best[c] < need) continue;
+        // exact check: prod(m) > 2 K (2^(in_bits-1) - 1)^2, all below 2^128
+        u128 prod = 1;
+        for (int t = 0; t < kNumWideModuli; ++t)
+            if (pick[c] >> t & 1) prod *= (u128)kWideModuli[t];
+        const u128 B = ((u128)1 << (in_bits - 1)) - 1;
+        const u128 bound = (u128)2 * (u128)K * B;  // prod > bound * B, written without forming bound * B
+        if (!(prod / B > bound || (prod / B == bound && prod % B != 0))) continue;
+        int n = 0;
+        for (int t = 0; t < kNumWideModuli; ++t)
+            if (pick[c] >> t & 1) out[n++] = kWideModuli[t];
+        return n;
+    }
+    return 0;
 }
 
 struct WideLayout {
@@ -215,14 +255,14 @@ extern "C" size_t awe_wide_workspace_bytes(int64_t M, int64_t N, int64_t K) {
     return wide_layout(M, N, K, &w) ? w.total : 0;
 }
 
-extern "C" awe_status_t awe_wide_residues(awe_handle_t h, const int64_t* X_dev, int64_t count, int8_t* res_dev,
-                                          void* stream) {
+static awe_status_t launch_residues(awe_handle_t h, const int64_t* X_dev, int64_t count, const int* moduli, int n,
+                                    int8_t* res_dev, void* stream) {
     if (!h || !X_dev || !res_dev || count <= 0) return AWE_ERR_INVALID_ARG;
     if ((uintptr_t)X_dev % 16 || (uintptr_t)res_dev % 4) return AWE_ERR_ALIGNMENT;
     ResidueParams p = {};
-    p.n = kNumWideModuli;
-    for (int t = 0; t < kNumWideModuli; ++t) {
-        const unsigned int m = (unsigned int)kWideModuli[t];
+    p.n = n;
+    for (int t = 0; t < n; ++t) {
+        const unsigned int m = (unsigned int)moduli[t];
         p.m[t] = (int)m;
         p.c1[t] = (1u << 14) % m;
         p.c2[t] = (1u << 28) % m;
@@ -237,12 +277,17 @@ extern "C" awe_status_t awe_wide_residues(awe_handle_t h, const int64_t* X_dev, 
     return AWE_OK;
 }
 
-extern "C" awe_status_t awe_wide_crt(awe_handle_t h, const int16_t* res_dev, int64_t count, int64_t* out_dev,
-                                     void* stream) {
+extern "C" awe_status_t awe_wide_residues(awe_handle_t h, const int64_t* X_dev, int64_t count, int8_t* res_dev,
+                                          void* stream) {
+    return launch_residues(h, X_dev, count, kWideModuli, kNumWideModuli, res_dev, stream);
+}
+
+static awe_status_t launch_crt(awe_handle_t h, const int16_t* res_dev, int64_t count, const int* moduli, int n,
+                               int64_t* out_dev, void* stream) {
     if (!h || !res_dev || !out_dev || count <= 0) return AWE_ERR_INVALID_ARG;
     if ((uintptr_t)res_dev % 2 || (uintptr_t)out_dev % 16) return AWE_ERR_ALIGNMENT;
     CrtParams c = {};
-    if (!build_crt_params(&c)) return AWE_ERR_UNSUPPORTED;
+    if (!build_crt_params(moduli, n, &c)) return AWE_ERR_UNSUPPORTED;
     const unsigned blocks = (unsigned)std::min<long long>((count + 255) / 256, (long long)h->sm_count * 16);
     wide_crt_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const short*)res_dev, count, c, (long long*)out_dev);
     if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
@@ -250,14 +295,30 @@ extern "C" awe_status_t awe_wide_crt(awe_handle_t h, const int16_t* res_dev, int
     return AWE_OK;
 }
 
+extern "C" awe_status_t awe_wide_crt(awe_handle_t h, const int16_t* res_dev, int64_t count, int64_t* out_dev,
+                                     void* stream) {
+    return launch_crt(h, res_dev, count, kWideModuli, kNumWideModuli, out_dev, stream);
+}
+
+extern "C" int awe_wide_select(int in_bits, int64_t K, int32_t* out, int capacity) {
+    if (in_bits < 2 || in_bits > 54 || K <= 0) return 0;
+    int sel[kMaxModuli];
+    const int n = select_moduli(in_bits, K, sel);
+    if (out)
+        for (int t = 0; t < n && t < capacity; ++t) out[t] = sel[t];
+    return n;
+}
+
 extern "C" awe_status_t awe_gemm_exact_wide(awe_handle_t h, const int64_t* A_dev, const int64_t* B_dev, int64_t M,
                                             int64_t N, int64_t K, int in_bits, int64_t* C_dev, void* workspace_dev,
                                             size_t workspace_bytes, void* stream) {
     if (!h || !A_dev || !B_dev || !C_dev || !workspace_dev || M <= 0 || N <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
     if (in_bits < 2 || in_bits > 54) return AWE_ERR_INVALID_ARG;
-    // unique reconstruction: prod(m) > 2 K B^2 with B = 2^(in_bits-1) - 1  (Section 5.3)
-    if (1.0L + log2l((long double)K) + 2.0L * (long double)(in_bits - 1) >= log2_of_moduli_product())
-        return AWE_ERR_RANGE;
+    // unique reconstruction: prod(m) > 2 K B^2 with B = 2^(in_bits-1) - 1  (Section 5.3); the cheapest
+    // subset of the built-in moduli that satisfies it is used
+    int sel[kMaxModuli];
+    const int n_sel = select_moduli(in_bits, K, sel);
+    if (n_sel == 0) return AWE_ERR_RANGE;
     WideLayout w;
     if (!wide_layout(M, N, K, &w)) return AWE_ERR_UNSUPPORTED;
     if (workspace_bytes < w.total) return AWE_ERR_WORKSPACE;
@@ -268,13 +329,13 @@ extern "C" awe_status_t awe_gemm_exact_wide(awe_handle_t h, const int64_t* A_dev
     int8_t* res_b = (int8_t*)(base + w.res_b);
     int16_t* res_c = (int16_t*)(base + w.res_c);
     awe_status_t s;
-    if ((s = awe_wide_residues(h, A_dev, M * K, res_a, stream)) != AWE_OK) return s;
-    if ((s = awe_wide_residues(h, B_dev, K * N, res_b, stream)) != AWE_OK) return s;
-    for (int t = 0; t < kNumWideModuli; ++t) {
+    if ((s = launch_residues(h, A_dev, M * K, sel, n_sel, res_a, stream)) != AWE_OK) return s;
+    if ((s = launch_residues(h, B_dev, K * N, sel, n_sel, res_b, stream)) != AWE_OK) return s;
+    for (int t = 0; t < n_sel; ++t) {
         s = awe_gemm_exact(h, res_a + (size_t)t * M * K, AWE_I8, res_b + (size_t)t * K * N, AWE_I8, M, N, K,
-                           AWE_ENC_MOD_M, kWideModuli[t], res_c + (size_t)t * M * N, AWE_C_RES_I16, base + w.planes,
+                           AWE_ENC_MOD_M, sel[t], res_c + (size_t)t * M * N, AWE_C_RES_I16, base + w.planes,
                            w.total - w.planes, stream);
         if (s != AWE_OK) return s;
     }
-    return awe_wide_crt(h, res_c, M * N, C_dev, stream);
+    return launch_crt(h, res_c, M * N, sel, n_sel, C_dev, stream);
 }

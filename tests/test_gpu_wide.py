@@ -82,6 +82,25 @@ def test_wide_product_equals_python_integers(shape):
     assert all(int(got[i]) == int(want[i]) for i in np.ndindex(M, N))
 
 
+@pytest.mark.parametrize("bits,K", [(32, 700), (24, 300), (12, 2000), (5, 64)])
+def test_narrower_inputs_use_a_cheaper_subset_and_stay_exact(bits, K):
+    h = gu.handle()
+    M, N = 70, 90
+    Bd = 2 ** (bits - 1) - 1
+    rng = np.random.default_rng(bits)
+    A = rng.integers(-Bd, Bd + 1, (M, K), dtype=np.int64)
+    B = rng.integers(-Bd, Bd + 1, (K, N), dtype=np.int64)
+    A[0, :], B[:, 0] = Bd, -Bd
+    sel = b.awe_wide_select(bits, K)
+    assert 0 < len(sel) < len(rns.RNS_SET_FP64)
+    ws = torch.empty(b.awe_wide_workspace_bytes(M, N, K), dtype=torch.uint8, device="cuda")
+    C = torch.zeros((M, N, 2), dtype=torch.int64, device="cuda")
+    b.awe_gemm_exact_wide(h, torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), M, N, K, bits, C, ws)
+    got = _to_python_ints(C.cpu().numpy())
+    want = rns.wide_matmul(A, B)
+    assert all(int(got[i]) == int(want[i]) for i in np.ndindex(M, N))
+
+
 def test_wide_product_agrees_with_the_oracle_pipeline_on_a_tiny_case():
     h = gu.handle()
     A, B = _wide_inputs(4, 3, 6, seed=5)

@@ -90,6 +90,21 @@ def test_sizes_and_host_side_rejections(b):
     assert "workspace" in b.status_string(3)
 
 
+def test_modulus_selection_matches_the_integer_program(b):
+    """awe_wide_select against the oracle's integer program restricted to the built-in moduli."""
+    import math
+    costs = {m: sc.mod_scheme(m).r for m in rns.RNS_SET_FP64}
+    for width, K in [(54, 16384), (54, 59000), (32, 8192), (24, 4096), (12, 1024), (9, 100000), (2, 1)]:
+        sel = b.awe_wide_select(width, K)
+        want_cost, _ = rns.select_moduli(costs, width=width, K=K)
+        B = 2 ** (width - 1) - 1
+        assert set(sel) <= set(rns.RNS_SET_FP64) and len(set(sel)) == len(sel)
+        assert math.prod(sel) > 2 * K * B * B
+        assert sum(costs[m] for m in sel) == want_cost, (width, K, sel)
+    assert b.awe_wide_select(54, 16384) == list(rns.RNS_SET_FP64)       # the full set is needed there
+    assert b.awe_wide_select(54, 70000) == []                           # beyond the built-in set
+
+
 def test_header_is_plain_c():
     """include/awe.h must compile as C (no C++ in the boundary)."""
     import subprocess
