@@ -506,7 +506,9 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
                                         const void* planesB_dev, int64_t M, int64_t N, int64_t K, void* C_dev,
                                         awe_out_dtype_t out_dt, int64_t ldc, int64_t k_chunk, void* stream) {
     if (!h || !planesA_dev || !planesB_dev || !C_dev || M <= 0 || N <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
-    if (M > (1 << 30) || N > (1 << 30) || K > (1ll << 36)) return AWE_ERR_INVALID_ARG;
+    // 32-bit tile counters and TMA coordinates: at most 2^31 bytes along a plane row and 2^30 tiles
+    if (M > (1 << 30) || N > (1 << 30) || K > (1ll << 31)) return AWE_ERR_INVALID_ARG;
+    if (((M + 127) / 128) * ((N + 127) / 128) > (1ll << 30)) return AWE_ERR_INVALID_ARG;
     if (ldc < N || k_chunk < 0 || (k_chunk % 256) != 0) return AWE_ERR_INVALID_ARG;
     if ((int)out_dt < 0 || (int)out_dt > 3) return AWE_ERR_INVALID_ARG;
     awe_encoding_desc d;
