@@ -65,9 +65,13 @@ typedef enum {
                                    (Section 6.2), K* = 2,097,152                                       */
     AWE_ENC_INT4xINT4_3 = 7,    /* INT4xINT4, 3 products (count from Section 5.2; the encoding is not
                                    printed: planes a0, a1, a0-a1 with weights (1,3))                  */
-    AWE_ENC_FP16SIG_AWE12 = 8   /* width-12 integers (FP16 significands with sign, |x| <= 2047; the
+    AWE_ENC_FP16SIG_AWE12 = 8,  /* width-12 integers (FP16 significands with sign, |x| <= 2047; the
                                    table also covers -2048), 12 products, w = v = (1,9,71,639), D = 2
                                    (Appendix A).  16-bit inputs (AWE_I16); 64-bit reconstruction.     */
+    AWE_ENC_INT8_MIXED_FP8_3 = 9 /* INT8xINT8 with 2 FP8 products and 1 FP4 product (Appendix A):
+                                   x = 13 h + 5 eps, planes h and h + eps stored as E4M3 bytes
+                                   (|.| <= 14), eps in S (|eps| <= 8) as E2M1;
+                                   xy = 104 hh' + 65 (h+eps)(h'+eps') - 40 eps eps', K* = 85,598.     */
 } awe_encoding_t;
 
 typedef enum {
@@ -108,6 +112,9 @@ typedef struct {
     int32_t c_a, c_b;               /* largest |stored plane value| per side (Section 3.4)       */
     int64_t k_star;                 /* floor(2^24 / (c_a c_b))                                   */
     int32_t a_lo, a_hi, b_lo, b_hi; /* input value range each side's table covers                */
+    int32_t plane_bits_a[AWE_MAX_PLANES]; /* storage width of each stored plane: 4 (E2M1) or 8 (E4M3) */
+    int32_t plane_bits_b[AWE_MAX_PLANES];
+    int32_t fp8[AWE_MAX_PRODUCTS];  /* 1 if product k multiplies E4M3 planes (an FP8 GEMM), else 0 */
 } awe_encoding_desc;
 
 /* Create / destroy a handle bound to CUDA device `device`.  awe_create makes that device
@@ -129,7 +136,9 @@ awe_status_t awe_encoding_lut(int enc, int modulus, awe_side_t side, awe_in_dtyp
 
 /* Bytes of the packed-plane buffer of one operand: n_planes x R x pitch, pitch =
  * round_up(K,256)/2 bytes (E2M1, two values per byte, even k in the low nibble, zero padded
- * along K).  0 on invalid arguments. */
+ * along K).  Planes stored as E4M3 (AWE_ENC_INT8_MIXED_FP8_3: planes 0 and 1) take one byte per
+ * value, i.e. rows of 2 x pitch bytes; plane j starts where plane j-1 ends.  0 on invalid
+ * arguments. */
 size_t awe_planes_bytes(int enc, int modulus, awe_side_t side, int64_t R, int64_t K);
 
 /* Bytes of scratch awe_gemm_exact needs (planes of A, then planes of B, each 256-B aligned). */
@@ -255,6 +264,15 @@ awe_status_t awe_gemm_exact_static(const void* A_dev, awe_in_dtype_t a_dt, const
  * P_dev: M x N float, leading dimension ldp.  The values returned are in the doubled-integer
  * convention of Section 3.1 (each operand counted as an element of S). */
 awe_status_t awe_fp4_product_raw(awe_handle_t h, const void* planeX_dev, const void* planeY_dev, int64_t M,
+                                 int64_t N, int64_t K, float* P_dev, int64_t ldp, void* stream);
+
+/* One raw FP8 (E4M3) product P = X.Y^T with FP32 accumulation over all of K in a single segment:
+ * the FP8 products of the mixed 2 x FP8 + 1 x FP4 construction (Appendix A) alone, so that a test
+ * can probe the exact-accumulation claim of Section 3.4 for this operand format too.
+ * planeX_dev: M x pitch8 bytes, planeY_dev: N x pitch8 bytes, pitch8 = round_up(K,256), one E4M3
+ * byte per element, zero-padded; both 256-byte aligned.  P_dev: M x N float, leading dimension
+ * ldp; values are the plain products (E4M3 holds the integers themselves, no doubling). */
+awe_status_t awe_fp8_product_raw(awe_handle_t h, const void* planeX_dev, const void* planeY_dev, int64_t M,
                                  int64_t N, int64_t K, float* P_dev, int64_t ldp, void* stream);
 
 /* Stand-alone reconstruction (Algorithm 1, last step; Section 5.3 for the residue form) from the r

@@ -22,6 +22,7 @@ ENC_INT8_AWE6, ENC_INT8_BASE13_9, ENC_INT4xINT8_AWE4, ENC_MOD_M, ENC_INT8_AWE6_A
 ENC_TERNARY_INT8_3 = 6
 ENC_INT4xINT4_3 = 7
 ENC_FP16SIG_AWE12 = 8
+ENC_INT8_MIXED_FP8_3 = 9
 I8, I4_IN_I8, T2_IN_I8, I16 = 0, 1, 2, 3
 C_I32, C_I64, C_RES_I16, C_RES_I32 = 0, 1, 2, 3
 SIDE_A, SIDE_B = 0, 1
@@ -32,7 +33,7 @@ STATIC_WORKSPACE_BYTES = 24 << 20
 EXPORTS = ["awe_create", "awe_destroy", "awe_encoding_info", "awe_encoding_lut", "awe_planes_bytes",
            "awe_workspace_bytes", "awe_host_staging_bytes", "awe_encode", "awe_gemm_planes", "awe_gemm_exact",
            "awe_gemm_exact_host", "awe_gemm_exact_static", "awe_wide_moduli", "awe_wide_select", "awe_wide_workspace_bytes",
-           "awe_wide_residues", "awe_wide_crt", "awe_gemm_exact_wide", "awe_reconstruct", "awe_fp4_product_raw", "awe_last_device_status", "awe_selftest_bounded_wait", "awe_last_gemm_clock_mhz", "awe_launch_count",
+           "awe_wide_residues", "awe_wide_crt", "awe_gemm_exact_wide", "awe_reconstruct", "awe_fp4_product_raw", "awe_fp8_product_raw", "awe_last_device_status", "awe_selftest_bounded_wait", "awe_last_gemm_clock_mhz", "awe_launch_count",
            "awe_status_string"]
 
 
@@ -42,7 +43,8 @@ class EncodingDesc(ctypes.Structure):
                 ("ell", ctypes.c_int32 * MAX_PRODUCTS), ("log2D", ctypes.c_int32), ("modulus", ctypes.c_int32),
                 ("c_a", ctypes.c_int32), ("c_b", ctypes.c_int32), ("k_star", ctypes.c_int64),
                 ("a_lo", ctypes.c_int32), ("a_hi", ctypes.c_int32), ("b_lo", ctypes.c_int32),
-                ("b_hi", ctypes.c_int32)]
+                ("b_hi", ctypes.c_int32), ("plane_bits_a", ctypes.c_int32 * MAX_PLANES),
+                ("plane_bits_b", ctypes.c_int32 * MAX_PLANES), ("fp8", ctypes.c_int32 * MAX_PRODUCTS)]
 
 
 class AweError(RuntimeError):
@@ -87,6 +89,7 @@ def lib() -> ctypes.CDLL:
     L.awe_gemm_exact_wide.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, sz, vp]
     L.awe_reconstruct.argtypes = [vp, i32, i32, vp, i64, i64, i64, i64, vp, i32, i64, vp]
     L.awe_fp4_product_raw.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
+    L.awe_fp8_product_raw.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
     L.awe_last_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.awe_selftest_bounded_wait.argtypes = [vp, i64, vp]
     L.awe_last_gemm_clock_mhz.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
@@ -261,6 +264,11 @@ def awe_gemm_exact_wide(h: Handle, A, B, M: int, N: int, K: int, in_bits: int, C
 def awe_fp4_product_raw(h: Handle, planeX, planeY, M: int, N: int, K: int, P, ldp: int, stream=None) -> None:
     _check(lib().awe_fp4_product_raw(h.raw, _ptr(planeX), _ptr(planeY), M, N, K, _ptr(P), ldp, _stream(stream)),
            "awe_fp4_product_raw")
+
+
+def awe_fp8_product_raw(h: Handle, planeX, planeY, M: int, N: int, K: int, P, ldp: int, stream=None) -> None:
+    _check(lib().awe_fp8_product_raw(h.raw, _ptr(planeX), _ptr(planeY), M, N, K, _ptr(P), ldp, _stream(stream)),
+           "awe_fp8_product_raw")
 
 
 def awe_reconstruct(h: Handle, enc: int, modulus: int, P, plane_stride: int, ldp: int, M: int, N: int, C,

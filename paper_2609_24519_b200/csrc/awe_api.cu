@@ -101,7 +101,10 @@ awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_i
 }
 }  // namespace awe
 
-static int t_planes(const awe_encoding_desc& d, awe_side_t side) { return side == AWE_SIDE_A ? d.n_planes_a : d.n_planes_b; }
+// rows of all stored planes of a side, in units of the E2M1 pitch (an E4M3 plane counts twice)
+static int t_planes(const awe_encoding_desc& d, awe_side_t side) {
+    return side == AWE_SIDE_A ? plane_units(d.plane_bits_a, d.n_planes_a) : plane_units(d.plane_bits_b, d.n_planes_b);
+}
 
 static size_t out_elem_bytes(awe_out_dtype_t t) { return t == AWE_C_I64 ? 8 : (t == AWE_C_RES_I16 ? 2 : 4); }
 

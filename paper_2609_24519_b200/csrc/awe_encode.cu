@@ -117,9 +117,46 @@ __device__ __forceinline__ void encode32_store(const unsigned char* lut_s, uint3
         *reinterpret_cast<uint4*>(dst + j * plane_stride) = make_uint4(o[0][j], o[1][j], o[2][j], o[3][j]);
 }
 
+// Mixed-format record (2 x FP8 + 1 x FP4, Appendix A): the table word of an input byte carries the
+// E4M3 bytes of planes 0 and 1 in bytes 0 and 1 and the E2M1 code of plane 2 in the low nibble of
+// byte 2.  32 consecutive elements of a row give 32 bytes of each E4M3 plane and 16 of the E2M1
+// plane.  Plane 0 starts at `planes`, plane 1 after R rows of 2*pitch bytes, plane 2 after that.
+__device__ __forceinline__ void encode32_store_mixed(const unsigned char* lut_s, uint32_t slot,
+                                                     const uint32_t (&in)[8], uint8_t* planes, int64_t R, int64_t row,
+                                                     int64_t k0, int64_t pitch) {
+    uint32_t p0[8], p1[8], p2[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const uint32_t w0 = in[2 * g], w1 = in[2 * g + 1];
+        const uint32_t e0 = lookup<3, 0>(lut_s, slot, w0).x, e1 = lookup<3, 1>(lut_s, slot, w0).x;
+        const uint32_t e2 = lookup<3, 2>(lut_s, slot, w0).x, e3 = lookup<3, 3>(lut_s, slot, w0).x;
+        const uint32_t e4 = lookup<3, 0>(lut_s, slot, w1).x, e5 = lookup<3, 1>(lut_s, slot, w1).x;
+        const uint32_t e6 = lookup<3, 2>(lut_s, slot, w1).x, e7 = lookup<3, 3>(lut_s, slot, w1).x;
+        const uint32_t t01 = __byte_perm(e0, e1, 0x5140), t23 = __byte_perm(e2, e3, 0x5140);
+        const uint32_t t45 = __byte_perm(e4, e5, 0x5140), t67 = __byte_perm(e6, e7, 0x5140);
+        p0[2 * g] = __byte_perm(t01, t23, 0x5410);
+        p1[2 * g] = __byte_perm(t01, t23, 0x7632);
+        p0[2 * g + 1] = __byte_perm(t45, t67, 0x5410);
+        p1[2 * g + 1] = __byte_perm(t45, t67, 0x7632);
+        // E2M1 pairs: even k in the low nibble (byte 2 of the even word), odd k in the high nibble
+        const uint32_t q01 = (e0 >> 16) | ((e1 >> 12) & 0xF0u), q23 = (e2 >> 16) | ((e3 >> 12) & 0xF0u);
+        const uint32_t q45 = (e4 >> 16) | ((e5 >> 12) & 0xF0u), q67 = (e6 >> 16) | ((e7 >> 12) & 0xF0u);
+        p2[g] = __byte_perm(__byte_perm(q01, q23, 0x0040), __byte_perm(q45, q67, 0x0040), 0x5410);
+    }
+    const int64_t pitch8 = 2 * pitch;
+    uint8_t* d0 = planes + row * pitch8 + k0;
+    uint8_t* d1 = d0 + R * pitch8;
+    uint8_t* d2 = planes + 2 * R * pitch8 + row * pitch + k0 / 2;
+    *reinterpret_cast<uint4*>(d0) = make_uint4(p0[0], p0[1], p0[2], p0[3]);
+    *reinterpret_cast<uint4*>(d0 + 16) = make_uint4(p0[4], p0[5], p0[6], p0[7]);
+    *reinterpret_cast<uint4*>(d1) = make_uint4(p1[0], p1[1], p1[2], p1[3]);
+    *reinterpret_cast<uint4*>(d1 + 16) = make_uint4(p1[4], p1[5], p1[6], p1[7]);
+    *reinterpret_cast<uint4*>(d2) = make_uint4(p2[0], p2[1], p2[2], p2[3]);
+}
+
 // Operand stored with the reduction index contiguous (A as M x K): a warp handles 1024
-// consecutive k of one row, 32 per lane.
-template <int NP>
+// consecutive k of one row, 32 per lane.  kMixed: the mixed-format record above (NP = 3).
+template <int NP, bool kMixed = false>
 __global__ void __launch_bounds__(kEncThreads)
 encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld, const uint64_t* __restrict__ lut_g,
                   uint8_t* __restrict__ planes, int64_t pitch, int64_t plane_stride, int vec_ok) {
@@ -154,7 +191,8 @@ encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
                 in[i] = word;
             }
         }
-        encode32_store<NP>(lut_s, slot, in, planes + row * pitch + k0 / 2, plane_stride);
+        if (kMixed) encode32_store_mixed(lut_s, slot, in, planes, R, row, k0, pitch);
+        else encode32_store<NP>(lut_s, slot, in, planes + row * pitch + k0 / 2, plane_stride);
     }
 }
 
@@ -165,7 +203,7 @@ encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
 // byte permutes into 4 rows of 32 consecutive k, and encodes each row exactly like the kernel
 // above.  The lanes of a group write adjacent 16-byte pieces in the same instruction, so whole
 // 32-byte sectors are written at once (a sector left half written costs a fill from DRAM).
-template <int NP>
+template <int NP, bool kMixed = false>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kxr_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld, const uint64_t* __restrict__ lut_g,
                   uint8_t* __restrict__ planes, int64_t pitch, int64_t plane_stride, int vec_ok) {
@@ -211,8 +249,11 @@ encode_kxr_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
             t[3][g] = __byte_perm(ab_hi, cd_hi, 0x7632);
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (r0 + j < R) encode32_store<NP>(lut_s, slot, t[j], planes + (r0 + j) * pitch + k0 / 2, plane_stride);
+        for (int j = 0; j < 4; ++j) {
+            if (r0 + j >= R) continue;
+            if (kMixed) encode32_store_mixed(lut_s, slot, t[j], planes, R, r0 + j, k0, pitch);
+            else encode32_store<NP>(lut_s, slot, t[j], planes + (r0 + j) * pitch + k0 / 2, plane_stride);
+        }
     }
 }
 
@@ -377,7 +418,7 @@ cudaError_t launch16(awe_layout_t layout, const uint16_t* X, int64_t R, int64_t 
     return cudaGetLastError();
 }
 
-template <int NP>
+template <int NP, bool kMixed = false>
 cudaError_t launch(awe_layout_t layout, const int8_t* X, int64_t R, int64_t K, int64_t ld, const uint64_t* lut,
                    uint8_t* planes, int64_t pitch, int64_t plane_stride, int vec_ok, int sm_count,
                    cudaStream_t stream) {
@@ -385,13 +426,13 @@ cudaError_t launch(awe_layout_t layout, const int8_t* X, int64_t R, int64_t K, i
     if (layout == AWE_ROWMAJOR_RxK) {
         const int64_t items = R * ((pitch * 2 + 1023) / 1024);
         const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
-        encode_rxk_kernel<NP><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(X, R, K, ld, lut, planes,
-                                                                                        pitch, plane_stride, vec_ok);
+        encode_rxk_kernel<NP, kMixed><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
+            X, R, K, ld, lut, planes, pitch, plane_stride, vec_ok);
     } else {
         const int64_t items = ((pitch * 2 + kKxrK - 1) / kKxrK) * ((R + kKxrRows - 1) / kKxrRows);
         const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
-        encode_kxr_kernel<NP><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(X, R, K, ld, lut, planes,
-                                                                                        pitch, plane_stride, vec_ok);
+        encode_kxr_kernel<NP, kMixed><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
+            X, R, K, ld, lut, planes, pitch, plane_stride, vec_ok);
     }
     return cudaGetLastError();
 }
@@ -433,6 +474,12 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
         return AWE_OK;
     }
     const int8_t* X = (const int8_t*)X_dev;
+    if (t->bits[0] == 8) {
+        e = launch<3, true>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st);
+        if (e != cudaSuccess) return AWE_ERR_CUDA;
+        h->launches += 1;
+        return AWE_OK;
+    }
     switch (t->n_planes) {
         case 1: e = launch<1>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st); break;
         case 2: e = launch<2>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st); break;

@@ -49,6 +49,9 @@ struct Cfg {
     // mxf4 instruction descriptor: E2M1 x E2M1, both K-major, UE8M0 scales, dense K = 64
     static constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | (1u << 23) |
                                        ((uint32_t)((kTileM * kCtas) >> 4) << 24);
+    // f8f6f4 instruction descriptor: E4M3 x E4M3 (format code 0), FP32 accumulator, both K-major, K = 32
+    static constexpr uint32_t kIdescF8 =
+        (1u << 4) | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)((kTileM * kCtas) >> 4) << 24);
 };
 constexpr int kMaxStages = 6;
 // Two accumulators of 256 columns and 32 columns of scale bytes do not fit 512 columns side by
@@ -145,10 +148,15 @@ __device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128]
     }
 }
 
-template <bool kPair>
+// kMixed: some products of the record multiply E4M3 planes (their own pair of tensor maps, 128
+// elements per 128-byte K block, kind::f8f6f4 without block scales, accumulator = the product
+// itself); the others are E2M1 products as above.  Pair variant only.
+template <bool kPair, bool kMixed>
 __global__ void __launch_bounds__(kThreads, 1)
 awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const __grid_constant__ CUtensorMap map_a8, const __grid_constant__ CUtensorMap map_b8,
                 const __grid_constant__ GemmParams p) {
+    static_assert(kPair || !kMixed, "mixed-format records run on CTA pairs");
     using C = Cfg<kPair>;
     constexpr int kStages = C::kStages;
     constexpr int kStageBytes = C::kStageBytes;
@@ -178,6 +186,10 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&map_a);
         ptx::prefetch_tensormap(&map_b);
+        if (kMixed) {
+            ptx::prefetch_tensormap(&map_a8);
+            ptx::prefetch_tensormap(&map_b8);
+        }
     }
     if (warp == 1) {
         if (kPair) {
@@ -215,6 +227,7 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int chunks = (p.num_kblocks + p.chunk_kblocks - 1) / p.chunk_kblocks;
+    const int chunks8 = kMixed ? (p.num_kblocks8 + p.chunk_kblocks8 - 1) / p.chunk_kblocks8 : 0;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -228,18 +241,22 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 const int row_b = tn * kTileN + (int)rank * C::kBRows;
                 for (int kk = 0; kk < p.r && ok; ++kk) {
                     const int k = product_at(kk, tile_iter, p.r);
-                    for (int kb = 0; kb < p.num_kblocks; ++kb, ++it) {
+                    const bool f8 = kMixed && p.fp8[k];
+                    const CUtensorMap* ma = f8 ? &map_a8 : &map_a;
+                    const CUtensorMap* mb = f8 ? &map_b8 : &map_b;
+                    const int nkb = f8 ? p.num_kblocks8 : p.num_kblocks, kb_first = f8 ? p.kblock0_8 : p.kblock0;
+                    for (int kb = 0; kb < nkb; ++kb, ++it) {
                         const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
                         if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->empty[s]), ph ^ 1u, p.status, 1))) break;
                         const uint32_t bar = ptx::smem_u32(&sh->full[s]);
                         const uint32_t a_dst = tiles_base + s * kStageBytes;
-                        const int x = (p.kblock0 + kb) * kBlockKBytes;
+                        const int x = (kb_first + kb) * kBlockKBytes;
                         if (kPair) {
                             // both CTAs report their bytes to CTA 0's barrier, which expects the sum
                             if (rank == 0) ptx::mbar_arrive_expect_tx(bar, 2 * kStageBytes);
                             const uint32_t bar0 = ptx::map_to_cta(bar, 0);
-                            ptx::tma_load_3d_pair(a_dst, &map_a, bar0, x, row_a, p.ia[k]);
-                            ptx::tma_load_3d_pair(a_dst + kABytes, &map_b, bar0, x, row_b, p.ib[k]);
+                            ptx::tma_load_3d_pair(a_dst, ma, bar0, x, row_a, p.ia[k]);
+                            ptx::tma_load_3d_pair(a_dst + kABytes, mb, bar0, x, row_b, p.ib[k]);
                         } else {
                             ptx::mbar_arrive_expect_tx(bar, kStageBytes);
                             ptx::tma_load_3d(a_dst, &map_a, bar, x, row_a, p.ia[k]);
@@ -254,9 +271,13 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // ---------------------------------------------------------------- MMA issuer
             uint32_t it = 0, drains = 0;
             bool ok = true;
-            for (int t = worker; t < num_tiles && ok; t += num_workers) {
-                for (int k = 0; k < p.r && ok; ++k) {
-                    for (int c = 0; c < chunks && ok; ++c, ++drains) {
+            for (int t = worker, tile_iter = 0; t < num_tiles && ok; t += num_workers, ++tile_iter) {
+                for (int kk = 0; kk < p.r && ok; ++kk) {
+                    const bool f8 = kMixed && p.fp8[product_at(kk, tile_iter, p.r)];
+                    const int nkb = f8 ? p.num_kblocks8 : p.num_kblocks;
+                    const int ckb = f8 ? p.chunk_kblocks8 : p.chunk_kblocks;
+                    const int nchunks = f8 ? chunks8 : chunks;
+                    for (int c = 0; c < nchunks && ok; ++c, ++drains) {
                         // accumulator (drains & 1): its previous contents (two segments ago) fully drained,
                         // and the columns it shares with the other accumulator already read
                         const uint32_t ab = drains & 1u;
@@ -268,8 +289,8 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             !(ok = bounded_wait(sh, ptx::smem_u32(&sh->overlap_free), (drains - 1u) & 1u, p.status, 5)))
                             break;
                         ptx::tc_fence_after();
-                        const int kb_end = min(p.num_kblocks, (c + 1) * p.chunk_kblocks);
-                        for (int kb = c * p.chunk_kblocks; kb < kb_end; ++kb, ++it) {
+                        const int kb_end = min(nkb, (c + 1) * ckb);
+                        for (int kb = c * ckb; kb < kb_end; ++kb, ++it) {
                             const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
                             if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->full[s]), ph, p.status, 3))) break;
                             ptx::tc_fence_after();
@@ -279,8 +300,10 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 // 64 elements = 32 bytes further along K inside the swizzle row
-                                const uint32_t acc = (kb > c * p.chunk_kblocks || j > 0) ? 1u : 0u;
-                                if (kPair)
+                                const uint32_t acc = (kb > c * ckb || j > 0) ? 1u : 0u;
+                                if (f8)
+                                    ptx::mma_f8_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, C::kIdescF8, acc);
+                                else if (kPair)
                                     ptx::mma_mxf4_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
                                                        tmem + kSfaCol, tmem + kSfbCol, acc);
                                 else
@@ -336,9 +359,13 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
             for (int i = 0; i < 128; ++i) sum[i] = 0;
             for (int kk = 0; kk < p.r && ok; ++kk) {
-                int ell = p.ell[product_at(kk, tile_iter, p.r)];
+                const int k = product_at(kk, tile_iter, p.r);
+                int ell = p.ell[k];
                 if (m && ell > m_hi) ell -= m;
-                for (int c = 0; c < chunks && ok; ++c, ++drains) {
+                const bool f8 = kMixed && p.fp8[k];
+                if (kMixed) em.acc_scale = f8 ? 1.0f : p.acc_scale;
+                const int nchunks = f8 ? chunks8 : chunks;
+                for (int c = 0; c < nchunks && ok; ++c, ++drains) {
                     const uint32_t ab = drains & 1u;
                     ok = bounded_wait(sh, ptx::smem_u32(&sh->acc_full[ab]), (drains >> 1) & 1u, p.status, 4);
                     ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below need the whole warp
@@ -450,13 +477,13 @@ bool use_pairs() {
     return v;
 }
 
-template <bool kPair>
-awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p,
-                            cudaStream_t st) {
+template <bool kPair, bool kMixed>
+awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ma8,
+                            const CUtensorMap& mb8, GemmParams& p, cudaStream_t st) {
     using C = Cfg<kPair>;
-    bool& attr_set = h->smem_attr_set[kPair ? 0 : 1];
+    bool& attr_set = h->smem_attr_set[kMixed ? 3 : (kPair ? 0 : 1)];
     if (!attr_set) {
-        if (cudaFuncSetAttribute(awe_gemm_kernel<kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(awe_gemm_kernel<kPair, kMixed>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)C::kSmemBytes) != cudaSuccess)
             return AWE_ERR_CUDA;
         attr_set = true;
@@ -478,7 +505,7 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair>, ma, mb, p);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair, kMixed>, ma, mb, ma8, mb8, p);
     if (err != cudaSuccess) {
         if (getenv("AWE_DEBUG")) fprintf(stderr, "awe: GEMM launch failed: %s\n", cudaGetErrorString(err));
         return AWE_ERR_CUDA;
@@ -488,7 +515,14 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
 }
 
 awe_status_t launch_gemm(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
-    return use_pairs() ? launch_variant<true>(h, ma, mb, p, st) : launch_variant<false>(h, ma, mb, p, st);
+    return use_pairs() ? launch_variant<true, false>(h, ma, mb, ma, mb, p, st)
+                       : launch_variant<false, false>(h, ma, mb, ma, mb, p, st);
+}
+
+// Records with E4M3 products: (ma, mb) cover the E2M1 planes, (ma8, mb8) the E4M3 planes.
+awe_status_t launch_gemm_mixed(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ma8,
+                               const CUtensorMap& mb8, GemmParams& p, cudaStream_t st) {
+    return launch_variant<true, true>(h, ma, mb, ma8, mb8, p, st);
 }
 
 int b_box_rows() { return use_pairs() ? Cfg<true>::kBRows : Cfg<false>::kBRows; }
@@ -530,19 +564,33 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
     static const bool force_wide = [] { const char* e = getenv("AWE_FORCE_WIDE_SUMS"); return e && e[0] == '1'; }();
     const bool wide = !residue && (force_wide || ((int64_t)1 << 30) / (amax * bmax * ((int64_t)1 << d.log2D)) < 256);
     if (wide && !use_pairs()) return AWE_ERR_UNSUPPORTED;
-    CUtensorMap ma, mb;
-    if ((s = make_plane_map(h, planesA_dev, M, pitch, d.n_planes_a, kTileM, &ma)) != AWE_OK) return s;
-    if ((s = make_plane_map(h, planesB_dev, N, pitch, d.n_planes_b, wide ? wide_b_box_rows() : b_box_rows(), &mb)) !=
+    // E4M3 planes (mixed-format records) come first in the buffer, with rows twice as long
+    int n8a = 0, n8b = 0;
+    while (n8a < d.n_planes_a && d.plane_bits_a[n8a] == 8) ++n8a;
+    while (n8b < d.n_planes_b && d.plane_bits_b[n8b] == 8) ++n8b;
+    const bool mixed = n8a > 0 || n8b > 0;
+    if (mixed && (wide || residue || !use_pairs() || n8a == d.n_planes_a || n8b == d.n_planes_b))
+        return AWE_ERR_UNSUPPORTED;
+    const uint8_t* a4 = (const uint8_t*)planesA_dev + (size_t)n8a * M * 2 * pitch;
+    const uint8_t* b4 = (const uint8_t*)planesB_dev + (size_t)n8b * N * 2 * pitch;
+    CUtensorMap ma, mb, ma8, mb8;
+    if ((s = make_plane_map(h, a4, M, pitch, d.n_planes_a - n8a, kTileM, &ma)) != AWE_OK) return s;
+    if ((s = make_plane_map(h, b4, N, pitch, d.n_planes_b - n8b, wide ? wide_b_box_rows() : b_box_rows(), &mb)) !=
         AWE_OK)
         return s;
+    if (mixed) {
+        if ((s = make_plane_map(h, planesA_dev, M, 2 * pitch, n8a, kTileM, &ma8)) != AWE_OK) return s;
+        if ((s = make_plane_map(h, planesB_dev, N, 2 * pitch, n8b, Cfg<true>::kBRows, &mb8)) != AWE_OK) return s;
+    }
 
     GemmParams p = {};
     p.M = (int)M;
     p.N = (int)N;
     p.r = d.r;
     for (int k = 0; k < d.r; ++k) {
-        p.ia[k] = d.ia[k];
-        p.ib[k] = d.ib[k];
+        p.fp8[k] = d.fp8[k];
+        p.ia[k] = d.fp8[k] ? d.ia[k] : d.ia[k] - n8a;  // index inside the map of its own format
+        p.ib[k] = d.fp8[k] ? d.ib[k] : d.ib[k] - n8b;
         p.ell[k] = d.ell[k];
     }
     p.log2D = d.log2D;
@@ -576,7 +624,16 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
         p.kblock0 = (int)kb0;
         p.num_kblocks = (int)std::min(seg_kblocks, total_kblocks - kb0);
         p.accumulate = kb0 > 0;
-        if ((s = launch_gemm(h, ma, mb, p, (cudaStream_t)stream)) != AWE_OK) return s;
+        if (mixed) {
+            // an E4M3 K block holds 128 elements, an E2M1 block 256
+            p.kblock0_8 = 2 * p.kblock0;
+            p.num_kblocks8 = 2 * p.num_kblocks;
+            p.chunk_kblocks8 = 2 * p.chunk_kblocks;
+            s = launch_gemm_mixed(h, ma, mb, ma8, mb8, p, (cudaStream_t)stream);
+        } else {
+            s = launch_gemm(h, ma, mb, p, (cudaStream_t)stream);
+        }
+        if (s != AWE_OK) return s;
     }
     return AWE_OK;
 }
@@ -616,4 +673,35 @@ extern "C" awe_status_t awe_fp4_product_raw(awe_handle_t h, const void* planeX_d
     p.num_kblocks = (int)(pitch / kBlockKBytes);
     p.chunk_kblocks = p.num_kblocks;
     return launch_gemm(h, ma, mb, p, (cudaStream_t)stream);
+}
+
+extern "C" awe_status_t awe_fp8_product_raw(awe_handle_t h, const void* planeX_dev, const void* planeY_dev,
+                                            int64_t M, int64_t N, int64_t K, float* P_dev, int64_t ldp,
+                                            void* stream) {
+    if (!h || !planeX_dev || !planeY_dev || !P_dev || M <= 0 || N <= 0 || K <= 0 || ldp < N)
+        return AWE_ERR_INVALID_ARG;
+    if (M > (1 << 30) || N > (1 << 30) || K > (1ll << 30)) return AWE_ERR_INVALID_ARG;
+    if ((uintptr_t)planeX_dev % 256 || (uintptr_t)planeY_dev % 256 || (uintptr_t)P_dev % 4) return AWE_ERR_ALIGNMENT;
+    if (!use_pairs()) return AWE_ERR_UNSUPPORTED;
+    const int64_t pitch8 = 2 * plane_pitch_bytes(K);
+    CUtensorMap ma, mb;
+    awe_status_t s;
+    if ((s = make_plane_map(h, planeX_dev, M, pitch8, 1, kTileM, &ma)) != AWE_OK) return s;
+    if ((s = make_plane_map(h, planeY_dev, N, pitch8, 1, Cfg<true>::kBRows, &mb)) != AWE_OK) return s;
+    GemmParams p = {};
+    p.M = (int)M;
+    p.N = (int)N;
+    p.r = 1;
+    p.ell[0] = 1;
+    p.fp8[0] = 1;
+    p.out_mode = OUT_RAW_F32;
+    p.C = P_dev;
+    p.ldc = ldp;
+    p.vec_store = ((uintptr_t)P_dev % 16 == 0) && ((ldp * 4) % 16 == 0);
+    p.acc_scale = kAccScale;
+    p.sf_word = kScaleWord;
+    p.num_kblocks = p.chunk_kblocks = 1;  // no E2M1 product in this launch
+    p.num_kblocks8 = (int)(pitch8 / kBlockKBytes);
+    p.chunk_kblocks8 = p.num_kblocks8;
+    return launch_gemm_mixed(h, ma, mb, ma, mb, p, (cudaStream_t)stream);
 }

@@ -30,6 +30,7 @@ struct SideTable {
     int n_planes = 0;
     int planes[AWE_MAX_PLANES][kMaxLimbs] = {{0}};
     int index_of_product[AWE_MAX_PRODUCTS] = {0};
+    int bits[AWE_MAX_PLANES] = {4, 4, 4, 4, 4, 4, 4, 4};  // storage width: 4 = E2M1 nibble, 8 = E4M3 byte
     int c = 0;       // largest |plane value| over the input range
     int entries = 0; // 256 (index: raw byte) or 4096 (index: low 12 bits of a 16-bit element)
     std::vector<int8_t> value;  // entries x AWE_MAX_PLANES plane values
@@ -44,6 +45,12 @@ awe_in_dtype_t natural_dtype(int enc, awe_side_t side);
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 inline int64_t plane_pitch_bytes(int64_t K) { return round_up(K, 256) / 2; }
 inline int64_t in_elem_bytes(awe_in_dtype_t dt) { return dt == AWE_I16 ? 2 : 1; }
+// Size of one row of all stored planes of a side, in units of the E2M1 pitch.
+inline int plane_units(const int32_t* bits, int n_planes) {
+    int u = 0;
+    for (int j = 0; j < n_planes; ++j) u += bits[j] / 4;
+    return u;
+}
 
 }  // namespace awe
 
@@ -69,7 +76,7 @@ struct awe_ctx {
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_done = nullptr;
     cudaEvent_t ev_a[kMaxHostChunks] = {nullptr}, ev_c[kMaxHostChunks] = {nullptr};
-    bool smem_attr_set[3] = {false, false, false};  // dynamic shared-memory limit raised (per kernel, this device)
+    bool smem_attr_set[4] = {false, false, false, false};  // dynamic shared-memory limit raised (per kernel, this device)
 };
 
 namespace awe {

@@ -152,6 +152,33 @@ Scheme make_fp16sig() {
     return s;
 }
 
+Scheme make_mixed_fp8() {
+    // x = 13 h + 5 eps on both sides; planes h, h + eps (E4M3) and eps (E2M1):
+    //   xy = 104 h h' + 65 (h + eps)(h' + eps') - 40 eps eps'                        (Appendix A)
+    Scheme s;
+    s.p = s.q = 2;
+    s.r = 3;
+    set_vec(s.w, {13, 5});
+    set_vec(s.v, {13, 5});
+    const int pl[3][2] = {{1, 0}, {1, 1}, {0, 1}};
+    for (int k = 0; k < 3; ++k)
+        for (int i = 0; i < 2; ++i) s.alpha[k][i] = s.beta[k][i] = pl[k][i];
+    set_vec(s.ell, {104, 65, -40});
+    return s;
+}
+
+// 8-bit E4M3 pattern (sign, 4 exponent bits with bias 7, 3 mantissa bits) of an integer |v| <= 15.
+uint8_t e4m3_code_of(int v) {
+    int a = std::abs(v);
+    if (a == 0) return 0;
+    int e = 0;
+    while ((a >> (e + 1)) != 0) ++e;             // a = 1.mmm x 2^e
+    const int mant = ((a << 3) >> e) & 7;        // exact for a <= 15
+    return (uint8_t)(((v < 0) ? 0x80 : 0) | ((e + 7) << 3) | mant);
+}
+
+constexpr int kFp8Cap = 14;  // largest |value| kept in an E4M3 plane (Appendix A: c_A = c_B = 14)
+
 struct Choice {
     int max_abs, sum_abs;
     int limbs[kMaxLimbs];
@@ -356,6 +383,10 @@ bool get_scheme(int enc, int modulus, Scheme* out) {
             s = make_ternary();
             ok = true;
             break;
+        case AWE_ENC_INT8_MIXED_FP8_3:
+            s = make_mixed_fp8();
+            ok = true;
+            break;
         case AWE_ENC_MOD_M:
             ok = make_mod(modulus, &s);
             break;
@@ -389,6 +420,40 @@ bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, co
     choose_tuples(n, weights, t.n_planes, t.planes, s.modulus, &best);
     const int lo = side == AWE_SIDE_A ? s.a_lo : s.b_lo;
     const int hi = side == AWE_SIDE_A ? s.a_hi : s.b_hi;
+    if (enc == AWE_ENC_INT8_MIXED_FP8_3) {
+        // Limb h is any integer whose planes h and h + eps fit E4M3 within +-14; eps in S, |eps| <= 8.
+        // Same choice rule as choose_tuples: largest |plane|, then sum of |planes|, then (h, eps).
+        if (dt != AWE_I8) return false;
+        t.bits[0] = t.bits[1] = 8;
+        t.c = 0;
+        for (int b = 0; b < 256; ++b) {
+            const int x = (int)(int8_t)b;
+            Choice best_c;
+            for (int e : kS) {
+                if (std::abs(e) > 8 || (x - 5 * e) % 13 != 0) continue;
+                Choice c;
+                const int hh = (x - 5 * e) / 13;
+                if (std::abs(hh) > kFp8Cap || std::abs(hh + e) > kFp8Cap) continue;
+                c.limbs[0] = hh;
+                c.limbs[1] = e;
+                c.max_abs = std::max(std::max(std::abs(hh), std::abs(hh + e)), std::abs(e));
+                c.sum_abs = std::abs(hh) + std::abs(hh + e) + std::abs(e);
+                c.valid = true;
+                if (better(c, best_c, 2)) best_c = c;
+            }
+            if (!best_c.valid) return false;
+            const int pv[3] = {best_c.limbs[0], best_c.limbs[0] + best_c.limbs[1], best_c.limbs[1]};
+            for (int j = 0; j < 3; ++j) {
+                t.value[(size_t)b * AWE_MAX_PLANES + j] = (int8_t)pv[j];
+                t.c = std::max(t.c, std::abs(pv[j]));
+            }
+            t.lut[b] = (uint64_t)e4m3_code_of(pv[0]) | ((uint64_t)e4m3_code_of(pv[1]) << 8) |
+                       ((uint64_t)e2m1_code_of(pv[2]) << 16);
+        }
+        auto ins_m = g_tables.emplace(key, t);
+        *out = &ins_m.first->second;
+        return true;
+    }
     t.c = 0;
     for (int b = 0; b < t.entries; ++b) {
         int x = (int)(int8_t)b;
@@ -448,6 +513,9 @@ extern "C" awe_status_t awe_encoding_info(int enc, int modulus, awe_encoding_des
     out->a_hi = s.a_hi;
     out->b_lo = s.b_lo;
     out->b_hi = s.b_hi;
+    for (int j = 0; j < ta->n_planes; ++j) out->plane_bits_a[j] = ta->bits[j];
+    for (int j = 0; j < tb->n_planes; ++j) out->plane_bits_b[j] = tb->bits[j];
+    for (int k = 0; k < s.r; ++k) out->fp8[k] = ta->bits[out->ia[k]] == 8;
     return AWE_OK;
 }
 
@@ -466,7 +534,7 @@ extern "C" size_t awe_planes_bytes(int enc, int modulus, awe_side_t side, int64_
     if (R <= 0 || K <= 0) return 0;
     const SideTable* t;
     if (!get_side_table(enc, modulus, side, natural_dtype(enc, side), &t)) return 0;
-    return (size_t)t->n_planes * (size_t)R * (size_t)plane_pitch_bytes(K);
+    return (size_t)plane_units(t->bits, t->n_planes) * (size_t)R * (size_t)plane_pitch_bytes(K);
 }
 
 extern "C" size_t awe_workspace_bytes(int enc, int modulus, int64_t M, int64_t N, int64_t K) {

@@ -39,6 +39,9 @@ struct GemmParams {
     int vec_store;     // C rows are 16-byte aligned: vector stores allowed
     float acc_scale;   // accumulator value -> product of doubled integers
     uint32_t sf_word;  // four copies of the UE8M0 scale byte
+    // Mixed-format records only: products whose planes are E4M3 bytes (128 elements per K block)
+    int fp8[AWE_MAX_PRODUCTS];
+    int kblock0_8, num_kblocks8, chunk_kblocks8;
 };
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
