@@ -338,6 +338,30 @@ def main():
         ctx["base13_9gemm_TOPS"] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
         ctx["base13_equals_awe6"] = bool(torch.equal(C9, C))
         del ws9, C9
+        # mixed 2 x FP8 + 1 x FP4 construction (Appendix A) on the same inputs: whole call and its product kernel
+        encm = b.ENC_INT8_MIXED_FP8_3
+        wsm = torch.empty(b.awe_workspace_bytes(encm, 0, M, N, K), dtype=torch.uint8, device=dev)
+        Cm = torch.empty_like(C)
+        for _ in range(3):
+            b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, encm, 0, Cm, b.C_I32, wsm)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(10):
+            b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, encm, 0, Cm, b.C_I32, wsm)
+        e1.record()
+        torch.cuda.synchronize()
+        ctx["mixed_2fp8_1fp4_TOPS"] = ops / (e0.elapsed_time(e1) / 10 * 1e-3) / 1e12
+        nAm = b.awe_planes_bytes(encm, 0, b.SIDE_A, M, K)
+        pam, pbm = wsm[:nAm], wsm[(nAm + 255) // 256 * 256:]
+        e0.record()
+        for _ in range(10):
+            b.awe_gemm_planes(h, encm, 0, pam, pbm, M, N, K, Cm, b.C_I32, N, 0)
+        e1.record()
+        torch.cuda.synchronize()
+        ctx["mixed_2fp8_1fp4_products_ms"] = e0.elapsed_time(e1) / 10
+        ctx["mixed_sm_mhz"] = b.awe_last_gemm_clock_mhz(h)
+        ctx["mixed_equals_awe6"] = bool(torch.equal(Cm, C))
+        del wsm, Cm, pam, pbm
         # INT8 tensor-core GEMM of the same product (library reference point)
         try:
             for _ in range(2):
