@@ -152,6 +152,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--size", type=int, default=8192, help="M = N = K of the headline workload")
+    ap.add_argument("--encoding", default="awe6", choices=["awe6", "awe6_alt", "base13", "mixed"],
+                    help="INT8xINT8 record of the timed step (the headline metric is awe6)")
     ap.add_argument("--no-extras", action="store_true", help="skip the context measurements")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     args = ap.parse_args()
@@ -186,7 +188,10 @@ def main():
         replicas.barrier(dev)
 
     h = b.awe_create(local_rank)
-    enc, M, N, K = b.ENC_INT8_AWE6, w.M, w.N, w.K
+    enc, enc_name = {"awe6": (b.ENC_INT8_AWE6, "int8_awe6"), "awe6_alt": (b.ENC_INT8_AWE6_ALT, "int8_awe6_alt"),
+                     "base13": (b.ENC_INT8_BASE13_9, "int8_base13_9"),
+                     "mixed": (b.ENC_INT8_MIXED_FP8_3, "int8_mixed_2fp8_1fp4")}[args.encoding]
+    M, N, K = w.M, w.N, w.K
     A, B = wl.make_inputs(w)
     dA, dB = torch.from_numpy(A).to(dev), torch.from_numpy(B).to(dev)
     C = torch.empty((M, N), dtype=torch.int32, device=dev)
@@ -272,12 +277,17 @@ def main():
     peaks = measured_peaks()
     fp4_peak = peaks["bf16_tflops_sustained"] * NOMINAL_FP4_OVER_BF16
     gemm_tflops = desc.r * ops / (ms_gemm * 1e-3) / 1e12
+    # an FP8 product runs at half the FP4 peak: the peak of a record is its flops over its ideal time
+    fp4_equiv = sum(2 if desc.fp8[k] else 1 for k in range(desc.r))
+    fmt_scale = desc.r / fp4_equiv  # 1 for FP4-only records
+    fp4_peak = fp4_peak * fmt_scale
     line = {
         "metric": METRIC, "value": ops_all_ranks / (ms_total * 1e-3) / 1e12, "unit": "TOPS", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "e2m1 (fp4) operands, f32 accumulate, int32 reconstruction",
         "data": "synthetic",
-        "config": {"workload": w.name, "M": M, "N": N, "K": K, "encoding": "int8_awe6", "fp4_gemms": desc.r,
+        "config": {"workload": w.name, "M": M, "N": N, "K": K, "encoding": enc_name, "fp4_gemms": desc.r - sum(desc.fp8[k] for k in range(desc.r)),
+                   "fp8_gemms": sum(desc.fp8[k] for k in range(desc.r)),
                    "inputs": "int8 uniform [-128,127], numpy default_rng(seed=6)", "output": "int32",
                    "l2": "no flush: per-step working set (64+64 MiB in, 384 MiB planes, 256 MiB out) exceeds the 126 MB L2",
                    "parallelism": "replicas only (no exchange step)" if world > 1 else "single GPU"},
@@ -288,16 +298,16 @@ def main():
         "parity": "3-call path == awe_gemm_exact == host path" if parity_ok else "MISMATCH between entry points",
         "kernels_ms": {"encode_a_plus_b": ms_encode, "gemm_and_reconstruction": ms_gemm},
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
-                     "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_BYTES_8192 if (M, N, K) == (8192, 8192, 8192) else None,
+                     "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_BYTES_8192 if (M, N, K, args.encoding) == (8192, 8192, 8192, "awe6") else None,
                      "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one launch at this workload "
                                      "(ncu capture with one-pass metrics; summary kept under profiles/)",
                      "kernel": "awe_gemm_kernel", "flops_per_launch": desc.r * ops,
                      "peak_source": "%s bf16 sustained %.1f TFLOP/s x nominal fp4:bf16 ratio 4" %
                                     (peaks["source"], peaks["bf16_tflops_sustained"]),
-                     "frac_of_nominal_9pflops": gemm_tflops / NOMINAL_FP4_TFLOPS,
+                     "frac_of_nominal_9pflops": gemm_tflops / (NOMINAL_FP4_TFLOPS * fmt_scale),
                      "frac_of_pipe_peak_at_delivered_clock":
-                         gemm_tflops / (MAC_PER_CLK_PER_SM * 2 * sm_count * gemm_mhz * 1e6 / 1e12) if gemm_mhz else None,
-                     "frac_of_burst_peak": gemm_tflops / (peaks["bf16_tflops"] * NOMINAL_FP4_OVER_BF16)},
+                         gemm_tflops / (fmt_scale * MAC_PER_CLK_PER_SM * 2 * sm_count * gemm_mhz * 1e6 / 1e12) if gemm_mhz else None,
+                     "frac_of_burst_peak": gemm_tflops / (peaks["bf16_tflops"] * NOMINAL_FP4_OVER_BF16 * fmt_scale)},
         "encode_roofline": {"bound": "hbm", "achieved": (M * K + K * N) * (1 + desc.n_planes_a / 2.0) / (ms_encode * 1e-3) / 1e9,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s"},
     }
@@ -487,7 +497,7 @@ def main():
             ceil_tflops = 2.0 * 8192 * 8192 * kz / (e0.elapsed_time(e1) / 10 * 1e-3) / 1e12
             ctx["fp4_ceiling_zero_data_TFLOPs"] = ceil_tflops
             ctx["fp4_ceiling_clock_mhz"] = b.awe_last_gemm_clock_mhz(h)
-            line["roofline"]["frac_of_measured_fp4_ceiling"] = gemm_tflops / ceil_tflops
+            line["roofline"]["frac_of_measured_fp4_ceiling"] = gemm_tflops / (ceil_tflops * fmt_scale)
             del pz
             # stand-alone reconstruction (HBM pass): 6 FP32 product matrices -> int32
             P6 = torch.zeros((6, 8192, 8192), dtype=torch.float32, device=dev)

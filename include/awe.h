@@ -78,8 +78,11 @@ typedef enum {
     AWE_I8 = 0,      /* one signed 8-bit value per byte                                          */
     AWE_I4_IN_I8 = 1, /* one signed 4-bit value per byte; only the low nibble is read (sign-extended) */
     AWE_T2_IN_I8 = 2, /* one ternary value -1, 0 or +1 per byte; any other byte is read as 0         */
-    AWE_I16 = 3       /* one signed 12-bit value per 16-bit element; only the low 12 bits are read
+    AWE_I16 = 3,      /* one signed 12-bit value per 16-bit element; only the low 12 bits are read
                          (sign-extended).  Leading dimensions stay in elements.                      */
+    AWE_I4_PACKED = 4 /* two signed 4-bit values per byte: element e of the row-major array sits in
+                         byte e/2, the even one in the low nibble.  Leading dimensions stay in
+                         elements and must be even (every row starts on a byte boundary).            */
 } awe_in_dtype_t;
 
 typedef enum {

@@ -59,6 +59,7 @@ extern "C" awe_status_t awe_destroy(awe_handle_t h) {
 namespace awe {
 awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, cudaStream_t stream,
                         const uint64_t** out) {
+    dt = table_dtype(dt);
     if (dt == AWE_I16) {  // 4096-entry tables live in their own arena (absent in the allocation-free context)
         if (!h->lut16_arena_dev) return AWE_ERR_UNSUPPORTED;
         for (size_t i = 0; i < h->slots16.size(); ++i)
@@ -111,8 +112,8 @@ static size_t out_elem_bytes(awe_out_dtype_t t) { return t == AWE_C_I64 ? 8 : (t
 extern "C" size_t awe_host_staging_bytes(int enc, int modulus, int64_t M, int64_t N, int64_t K,
                                          awe_out_dtype_t out_dt) {
     if (!awe_workspace_bytes(enc, modulus, M, N, K)) return 0;
-    const int64_t ea = in_elem_bytes(natural_dtype(enc, AWE_SIDE_A)), eb = in_elem_bytes(natural_dtype(enc, AWE_SIDE_B));
-    return (size_t)round_up(M * K * ea, 256) + (size_t)round_up(K * N * eb, 256) +
+    const awe_in_dtype_t na = natural_dtype(enc, AWE_SIDE_A), nb = natural_dtype(enc, AWE_SIDE_B);
+    return (size_t)round_up(in_bytes(na, M * K), 256) + (size_t)round_up(in_bytes(nb, K * N), 256) +
            (size_t)round_up(M * N * (int64_t)out_elem_bytes(out_dt), 256);
 }
 
@@ -163,12 +164,14 @@ extern "C" awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, 
     if ((uintptr_t)scratch_dev % 256) return AWE_ERR_ALIGNMENT;
     cudaStream_t st = (cudaStream_t)stream;
     uint8_t* base = (uint8_t*)scratch_dev;
-    const int64_t ea = in_elem_bytes(a_dt), eb = in_elem_bytes(b_dt);
-    if (ea != in_elem_bytes(natural_dtype(enc, AWE_SIDE_A)) || eb != in_elem_bytes(natural_dtype(enc, AWE_SIDE_B)))
+    // staging is sized for the natural container of the encoding; a packed 4-bit operand needs less
+    if (in_elem_nibbles(a_dt) > in_elem_nibbles(natural_dtype(enc, AWE_SIDE_A)) ||
+        in_elem_nibbles(b_dt) > in_elem_nibbles(natural_dtype(enc, AWE_SIDE_B)))
         return AWE_ERR_UNSUPPORTED;
+    if ((a_dt == AWE_I4_PACKED && (K & 1)) || (b_dt == AWE_I4_PACKED && (N & 1))) return AWE_ERR_INVALID_ARG;
     uint8_t* dA = base + round_up((int64_t)ws, 256);
-    uint8_t* dB = dA + round_up(M * K * ea, 256);
-    uint8_t* dC = dB + round_up(K * N * eb, 256);
+    uint8_t* dB = dA + round_up(in_bytes(natural_dtype(enc, AWE_SIDE_A), M * K), 256);
+    uint8_t* dC = dB + round_up(in_bytes(natural_dtype(enc, AWE_SIDE_B), K * N), 256);
     const size_t elem = out_elem_bytes(out_dt);
     // Everything awe_gemm_exact would reject is rejected here, before any copy is enqueued.
     awe_encoding_desc d;
@@ -205,7 +208,7 @@ extern "C" awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, 
     AWE_CU(cudaEventRecord(h->ev_start, st));
     AWE_CU(cudaStreamWaitEvent(h->copy_in, h->ev_start, 0));
     AWE_CU(cudaStreamWaitEvent(h->copy_out, h->ev_start, 0));
-    AWE_CU(cudaMemcpyAsync(dB, B_host, (size_t)K * N * eb, cudaMemcpyHostToDevice, h->copy_in));
+    AWE_CU(cudaMemcpyAsync(dB, B_host, (size_t)in_bytes(b_dt, K * N), cudaMemcpyHostToDevice, h->copy_in));
     AWE_CU(cudaEventRecord(h->ev_b, h->copy_in));
     AWE_CU(cudaStreamWaitEvent(st, h->ev_b, 0));
     if ((s = awe_encode(h, enc, modulus, AWE_SIDE_B, dB, b_dt, AWE_ROWMAJOR_KxR, N, K, N, pb, stream)) != AWE_OK) return s;
@@ -213,11 +216,11 @@ extern "C" awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, 
     int c = 0;
     for (int64_t r0 = 0; r0 < M; r0 += rows_per_chunk, ++c) {
         const int64_t rows = std::min(rows_per_chunk, M - r0);
-        const uint8_t* a_src = (const uint8_t*)A_host + (size_t)r0 * K * ea;
-        uint8_t* a_dst = dA + (size_t)r0 * K * ea;
+        const uint8_t* a_src = (const uint8_t*)A_host + (size_t)in_bytes(a_dt, r0 * K);
+        uint8_t* a_dst = dA + (size_t)in_bytes(a_dt, r0 * K);
         uint8_t* pa_c = pa + (size_t)t_planes(d, AWE_SIDE_A) * (size_t)r0 * pitch;  // this chunk's own plane block
         uint8_t* c_dst = dC + (size_t)r0 * N * elem;
-        AWE_CU(cudaMemcpyAsync(a_dst, a_src, (size_t)rows * K * ea, cudaMemcpyHostToDevice, h->copy_in));
+        AWE_CU(cudaMemcpyAsync(a_dst, a_src, (size_t)in_bytes(a_dt, rows * K), cudaMemcpyHostToDevice, h->copy_in));
         AWE_CU(cudaEventRecord(h->ev_a[c], h->copy_in));
         AWE_CU(cudaStreamWaitEvent(st, h->ev_a[c], 0));
         if ((s = awe_encode(h, enc, modulus, AWE_SIDE_A, a_dst, a_dt, AWE_ROWMAJOR_RxK, rows, K, K, pa_c, stream)) != AWE_OK)

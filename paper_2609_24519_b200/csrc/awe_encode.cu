@@ -156,7 +156,9 @@ __device__ __forceinline__ void encode32_store_mixed(const unsigned char* lut_s,
 
 // Operand stored with the reduction index contiguous (A as M x K): a warp handles 1024
 // consecutive k of one row, 32 per lane.  kMixed: the mixed-format record above (NP = 3).
-template <int NP, bool kMixed = false>
+// kPacked: the operand holds two 4-bit values per byte (element e of the array in byte e/2, low
+// nibble first); nibbles are spread to one per byte and then take the same route.
+template <int NP, bool kMixed = false, bool kPacked = false>
 __global__ void __launch_bounds__(kEncThreads)
 encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld, const uint64_t* __restrict__ lut_g,
                   uint8_t* __restrict__ planes, int64_t pitch, int64_t plane_stride, int vec_ok) {
@@ -172,8 +174,31 @@ encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
         const int64_t row = it / chunks, k0 = (it % chunks) * 1024 + lane * 32;
         if (k0 >= Kp) continue;
         uint32_t in[8];
-        const int8_t* src = X + row * ld + k0;
-        if (vec_ok && k0 + 32 <= K) {
+        const int8_t* src = kPacked ? X + (row * ld + k0) / 2 : X + row * ld + k0;
+        if (kPacked && vec_ok && k0 + 32 <= K) {
+            const uint4 a = __ldg(reinterpret_cast<const uint4*>(src));
+            const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t lo = w[i] & 0x0F0F0F0Fu, hi = (w[i] >> 4) & 0x0F0F0F0Fu;
+                in[2 * i] = __byte_perm(lo, hi, 0x5140);
+                in[2 * i + 1] = __byte_perm(lo, hi, 0x7362);
+            }
+        } else if (kPacked) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int64_t k = k0 + i * 4 + j;
+                    if (k < K) {
+                        const int64_t e = row * ld + k;
+                        word |= (((uint32_t)(uint8_t)X[e >> 1] >> (4 * (e & 1))) & 0xFu) << (8 * j);
+                    }
+                }
+                in[i] = word;
+            }
+        } else if (vec_ok && k0 + 32 <= K) {
             const uint4 a = __ldg(reinterpret_cast<const uint4*>(src));
             const uint4 b = __ldg(reinterpret_cast<const uint4*>(src) + 1);
             in[0] = a.x; in[1] = a.y; in[2] = a.z; in[3] = a.w;
@@ -203,7 +228,7 @@ encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
 // byte permutes into 4 rows of 32 consecutive k, and encodes each row exactly like the kernel
 // above.  The lanes of a group write adjacent 16-byte pieces in the same instruction, so whole
 // 32-byte sectors are written at once (a sector left half written costs a fill from DRAM).
-template <int NP, bool kMixed = false>
+template <int NP, bool kMixed = false, bool kPacked = false>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kxr_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld, const uint64_t* __restrict__ lut_g,
                   uint8_t* __restrict__ planes, int64_t pitch, int64_t plane_stride, int vec_ok) {
@@ -221,7 +246,28 @@ encode_kxr_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
         const int64_t k0 = (it / r_items) * kKxrK + (lane % kKxrLanesK) * 32;
         if (r0 >= R || k0 >= Kp) continue;
         uint32_t raw[32];  // raw[i] = bytes X[k0+i][r0..r0+3]
-        if (vec_ok && r0 + 4 <= R && k0 + 32 <= K) {
+        if (kPacked && vec_ok && r0 + 4 <= R && k0 + 32 <= K) {
+            // 4 elements = 2 bytes per k row
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const uint32_t w = __ldg(reinterpret_cast<const uint16_t*>(X + ((k0 + i) * ld + r0) / 2));
+                raw[i] = __byte_perm(w & 0x0F0Fu, (w >> 4) & 0x0F0Fu, 0x5140);
+            }
+        } else if (kPacked) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                uint32_t word = 0;
+                if (k0 + i < K) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (r0 + j < R) {
+                            const int64_t e = (k0 + i) * ld + r0 + j;
+                            word |= (((uint32_t)(uint8_t)X[e >> 1] >> (4 * (e & 1))) & 0xFu) << (8 * j);
+                        }
+                }
+                raw[i] = word;
+            }
+        } else if (vec_ok && r0 + 4 <= R && k0 + 32 <= K) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) raw[i] = __ldg(reinterpret_cast<const uint32_t*>(X + (k0 + i) * ld + r0));
         } else {
@@ -418,7 +464,7 @@ cudaError_t launch16(awe_layout_t layout, const uint16_t* X, int64_t R, int64_t 
     return cudaGetLastError();
 }
 
-template <int NP, bool kMixed = false>
+template <int NP, bool kMixed = false, bool kPacked = false>
 cudaError_t launch(awe_layout_t layout, const int8_t* X, int64_t R, int64_t K, int64_t ld, const uint64_t* lut,
                    uint8_t* planes, int64_t pitch, int64_t plane_stride, int vec_ok, int sm_count,
                    cudaStream_t stream) {
@@ -426,12 +472,12 @@ cudaError_t launch(awe_layout_t layout, const int8_t* X, int64_t R, int64_t K, i
     if (layout == AWE_ROWMAJOR_RxK) {
         const int64_t items = R * ((pitch * 2 + 1023) / 1024);
         const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
-        encode_rxk_kernel<NP, kMixed><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
+        encode_rxk_kernel<NP, kMixed, kPacked><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
             X, R, K, ld, lut, planes, pitch, plane_stride, vec_ok);
     } else {
         const int64_t items = ((pitch * 2 + kKxrK - 1) / kKxrK) * ((R + kKxrRows - 1) / kKxrRows);
         const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
-        encode_kxr_kernel<NP, kMixed><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
+        encode_kxr_kernel<NP, kMixed, kPacked><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
             X, R, K, ld, lut, planes, pitch, plane_stride, vec_ok);
     }
     return cudaGetLastError();
@@ -447,8 +493,9 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
                                    void* planes_dev, void* stream) {
     if (!h || !X_dev || !planes_dev || R <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
     if (side != AWE_SIDE_A && side != AWE_SIDE_B) return AWE_ERR_INVALID_ARG;
-    if ((int)dt < 0 || (int)dt > 3) return AWE_ERR_INVALID_ARG;
+    if ((int)dt < 0 || (int)dt > 4) return AWE_ERR_INVALID_ARG;
     if (layout != AWE_ROWMAJOR_RxK && layout != AWE_ROWMAJOR_KxR) return AWE_ERR_INVALID_ARG;
+    if (dt == AWE_I4_PACKED && (ld & 1)) return AWE_ERR_INVALID_ARG;  // rows start on byte boundaries
     if (ld < (layout == AWE_ROWMAJOR_RxK ? K : R)) return AWE_ERR_INVALID_ARG;
     if ((uintptr_t)planes_dev % 256) return AWE_ERR_ALIGNMENT;
     const SideTable* t;
@@ -474,6 +521,20 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
         return AWE_OK;
     }
     const int8_t* X = (const int8_t*)X_dev;
+    if (dt == AWE_I4_PACKED) {
+        // vector path: 16-byte loads of 32 nibbles along k (RxK) or 2-byte loads of 4 nibbles along r (KxR)
+        const int vp = layout == AWE_ROWMAJOR_RxK ? (((uintptr_t)X_dev % 16 == 0) && (ld % 32 == 0))
+                                                  : (((uintptr_t)X_dev % 2 == 0) && (ld % 4 == 0));
+        switch (t->n_planes) {
+            case 2: e = launch<2, false, true>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vp, h->sm_count, st); break;
+            case 3: e = launch<3, false, true>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vp, h->sm_count, st); break;
+            case 4: e = launch<4, false, true>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vp, h->sm_count, st); break;
+            default: return AWE_ERR_UNSUPPORTED;
+        }
+        if (e != cudaSuccess) return AWE_ERR_CUDA;
+        h->launches += 1;
+        return AWE_OK;
+    }
     if (t->bits[0] == 8) {
         e = launch<3, true>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st);
         if (e != cudaSuccess) return AWE_ERR_CUDA;

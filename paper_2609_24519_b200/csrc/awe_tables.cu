@@ -400,6 +400,7 @@ bool get_scheme(int enc, int modulus, Scheme* out) {
 }
 
 bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, const SideTable** out) {
+    dt = table_dtype(dt);
     Scheme s;
     if (!get_scheme(enc, modulus, &s)) return false;
     std::lock_guard<std::mutex> lock(g_mu);
@@ -521,7 +522,7 @@ extern "C" awe_status_t awe_encoding_info(int enc, int modulus, awe_encoding_des
 
 extern "C" awe_status_t awe_encoding_lut(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt,
                                          int8_t* lut_host) {
-    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (int)dt < 0 || (int)dt > 3)
+    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (int)dt < 0 || (int)dt > 4)
         return AWE_ERR_INVALID_ARG;
     const SideTable* t;
     if (!get_side_table(enc, modulus, side, dt, &t)) return AWE_ERR_UNSUPPORTED;
