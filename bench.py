@@ -277,6 +277,7 @@ def main():
     peaks = measured_peaks()
     fp4_peak = peaks["bf16_tflops_sustained"] * NOMINAL_FP4_OVER_BF16
     gemm_tflops = desc.r * ops / (ms_gemm * 1e-3) / 1e12
+    plane_bytes = b.awe_planes_bytes(enc, 0, b.SIDE_A, M, K) + b.awe_planes_bytes(enc, 0, b.SIDE_B, N, K)
     # an FP8 product runs at half the FP4 peak: the peak of a record is its flops over its ideal time
     fp4_equiv = sum(2 if desc.fp8[k] else 1 for k in range(desc.r))
     fmt_scale = desc.r / fp4_equiv  # 1 for FP4-only records
@@ -289,7 +290,8 @@ def main():
         "config": {"workload": w.name, "M": M, "N": N, "K": K, "encoding": enc_name, "fp4_gemms": desc.r - sum(desc.fp8[k] for k in range(desc.r)),
                    "fp8_gemms": sum(desc.fp8[k] for k in range(desc.r)),
                    "inputs": "int8 uniform [-128,127], numpy default_rng(seed=6)", "output": "int32",
-                   "l2": "no flush: per-step working set (64+64 MiB in, 384 MiB planes, 256 MiB out) exceeds the 126 MB L2",
+                   "l2": "no flush: per-step working set (%d+%d MiB in, %d MiB planes, %d MiB out) exceeds the 126 MB L2"
+                         % (M * K >> 20, K * N >> 20, plane_bytes >> 20, M * N * 4 >> 20),
                    "parallelism": "replicas only (no exchange step)" if world > 1 else "single GPU"},
         "clocks": clocks,
         "e2e": {"value": ops_e2e_all / (ms_e2e_total * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms_e2e,
@@ -308,13 +310,13 @@ def main():
                      "frac_of_pipe_peak_at_delivered_clock":
                          gemm_tflops / (fmt_scale * MAC_PER_CLK_PER_SM * 2 * sm_count * gemm_mhz * 1e6 / 1e12) if gemm_mhz else None,
                      "frac_of_burst_peak": gemm_tflops / (peaks["bf16_tflops"] * NOMINAL_FP4_OVER_BF16 * fmt_scale)},
-        "encode_roofline": {"bound": "hbm", "achieved": (M * K + K * N) * (1 + desc.n_planes_a / 2.0) / (ms_encode * 1e-3) / 1e9,
+        "encode_roofline": {"bound": "hbm", "achieved": (M * K + K * N + plane_bytes) / (ms_encode * 1e-3) / 1e9,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s"},
     }
     line["encode_roofline"]["frac"] = line["encode_roofline"]["achieved"] / peaks["hbm_gbs"]
     # The encode writes 3 bytes for every byte it reads, and HBM writes alone run well below the
     # read+write copy figure: measure a plain fill of the same size and report the write stream against it.
-    fill_buf = torch.empty(int((M * K + K * N) * desc.n_planes_a / 2), dtype=torch.uint8, device=dev)
+    fill_buf = torch.empty(plane_bytes, dtype=torch.uint8, device=dev)
     for _ in range(3):
         fill_buf.fill_(1)
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
