@@ -1,0 +1,88 @@
+"""Seeded random sweep: every encoding on random shapes (ragged tiles, tiny and odd sizes), random
+leading dimensions of C and random value mixes, against the plain int64 product of the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import matmul as mm
+from oracle import rns
+from paper_2609_24519_b200 import binding as b
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+# encoding, dtype and value range of A, dtype and value range of B
+KINDS = [
+    ("awe6", b.ENC_INT8_AWE6, b.I8, (-128, 127), b.I8, (-128, 127)),
+    ("awe6_alt", b.ENC_INT8_AWE6_ALT, b.I8, (-128, 127), b.I8, (-128, 127)),
+    ("base13", b.ENC_INT8_BASE13_9, b.I8, (-128, 127), b.I8, (-128, 127)),
+    ("mixed", b.ENC_INT8_MIXED_FP8_3, b.I8, (-128, 127), b.I8, (-128, 127)),
+    ("awe4", b.ENC_INT4xINT8_AWE4, b.I4_IN_I8, (-8, 7), b.I8, (-128, 127)),
+    ("int4x4", b.ENC_INT4xINT4_3, b.I4_IN_I8, (-8, 7), b.I4_IN_I8, (-8, 7)),
+    ("ternary", b.ENC_TERNARY_INT8_3, b.T2_IN_I8, (-1, 1), b.I8, (-128, 127)),
+    ("fp16sig", b.ENC_FP16SIG_AWE12, b.I16, (-2047, 2047), b.I16, (-2047, 2047)),
+]
+
+
+def _draw(rng, lo, hi, shape, dtype, style):
+    if style == 0:
+        X = rng.integers(lo, hi + 1, shape)
+    elif style == 1:                                   # extremes only
+        X = rng.choice(np.array([lo, hi]), shape)
+    elif style == 2:                                   # sparse: mostly zeros
+        X = rng.integers(lo, hi + 1, shape) * (rng.random(shape) < 0.1)
+    else:                                              # small magnitudes
+        X = rng.integers(max(lo, -2), min(hi, 2) + 1, shape)
+    return X.astype(dtype)
+
+
+@pytest.mark.parametrize("case", range(48))
+def test_random_shape_and_values(case):
+    rng = np.random.default_rng(1000 + case)
+    name, enc, a_dt, (alo, ahi), b_dt, (blo, bhi) = KINDS[case % len(KINDS)]
+    M, N = int(rng.integers(1, 700)), int(rng.integers(1, 700))
+    K = int(rng.integers(1, 3000))
+    np_dt = np.int16 if a_dt == b.I16 else np.int8
+    A = _draw(rng, alo, ahi, (M, K), np_dt, int(rng.integers(0, 4)))
+    B = _draw(rng, blo, bhi, (K, N), np_dt, int(rng.integers(0, 4)))
+    want = mm.matmul_i64_s16(A, B) if a_dt == b.I16 else mm.matmul_i64(A, B)
+    out_dt = b.C_I64 if (a_dt == b.I16 or case % 3 == 0) else b.C_I32
+    got = gu.gpu_gemm_exact(A, B, enc, out_dt, a_dt=a_dt, b_dt=b_dt)
+    assert np.array_equal(got.astype(np.int64), want), (name, M, N, K)
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_random_modulus_shape_and_values(case):
+    rng = np.random.default_rng(2000 + case)
+    m = int(rng.choice(np.array(rns.RNS_SET_FP64)))
+    M, N, K = int(rng.integers(1, 600)), int(rng.integers(1, 600)), int(rng.integers(1, 5000))
+    A = rng.integers(-128, 128, (M, K), dtype=np.int8)
+    B = rng.integers(-128, 128, (K, N), dtype=np.int8)
+    want = mm.mod_symmetric(mm.matmul_i64(A, B), m)
+    out_dt = b.C_RES_I16 if case % 2 else b.C_RES_I32
+    got = gu.gpu_gemm_exact(A, B, b.ENC_MOD_M, out_dt, modulus=m)
+    assert np.array_equal(got.astype(np.int64), want), (m, M, N, K)
+
+
+@pytest.mark.parametrize("case", range(8))
+def test_planes_entry_with_random_leading_dimension(case):
+    """awe_gemm_planes with ldc > N: the columns beyond N must stay untouched."""
+    rng = np.random.default_rng(3000 + case)
+    enc = [b.ENC_INT8_AWE6, b.ENC_INT8_MIXED_FP8_3][case % 2]
+    M, N, K = int(rng.integers(1, 500)), int(rng.integers(1, 500)), int(rng.integers(1, 2000))
+    ldc = N + int(rng.integers(0, 9))
+    A = rng.integers(-128, 128, (M, K), dtype=np.int8)
+    B = rng.integers(-128, 128, (K, N), dtype=np.int8)
+    h = gu.handle()
+    nA = b.awe_planes_bytes(enc, 0, b.SIDE_A, M, K)
+    ws = torch.empty(b.awe_workspace_bytes(enc, 0, M, N, K), dtype=torch.uint8, device="cuda")
+    pa, pb = ws[:nA], ws[(nA + 255) // 256 * 256:]
+    b.awe_encode(h, enc, 0, b.SIDE_A, torch.from_numpy(A).cuda(), b.I8, b.ROWMAJOR_RxK, M, K, K, pa)
+    b.awe_encode(h, enc, 0, b.SIDE_B, torch.from_numpy(B).cuda(), b.I8, b.ROWMAJOR_KxR, N, K, N, pb)
+    C = torch.full((M, ldc), 77, dtype=torch.int32, device="cuda")
+    b.awe_gemm_planes(h, enc, 0, pa, pb, M, N, K, C, b.C_I32, ldc, 0)
+    torch.cuda.synchronize()
+    assert b.awe_last_device_status(h) == (0, 0)
+    got = C.cpu().numpy()
+    assert np.array_equal(got[:, :N].astype(np.int64), mm.matmul_i64(A, B))
+    assert (got[:, N:] == 77).all()
