@@ -26,6 +26,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstdlib>
+#include <type_traits>
 
 #include "gemm_common.cuh"
 
@@ -242,8 +243,6 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 for (int kk = 0; kk < p.r && ok; ++kk) {
                     const int k = product_at(kk, tile_iter, p.r);
                     const bool f8 = kMixed && p.fp8[k];
-                    const CUtensorMap* ma = f8 ? &map_a8 : &map_a;
-                    const CUtensorMap* mb = f8 ? &map_b8 : &map_b;
                     const int nkb = f8 ? p.num_kblocks8 : p.num_kblocks, kb_first = f8 ? p.kblock0_8 : p.kblock0;
                     for (int kb = 0; kb < nkb; ++kb, ++it) {
                         const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
@@ -255,8 +254,15 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             // both CTAs report their bytes to CTA 0's barrier, which expects the sum
                             if (rank == 0) ptx::mbar_arrive_expect_tx(bar, 2 * kStageBytes);
                             const uint32_t bar0 = ptx::map_to_cta(bar, 0);
-                            ptx::tma_load_3d_pair(a_dst, ma, bar0, x, row_a, p.ia[k]);
-                            ptx::tma_load_3d_pair(a_dst + kABytes, mb, bar0, x, row_b, p.ib[k]);
+                            // each load names its tensor map directly (a pointer chosen at run time between
+                            // two kernel parameters made every copy far slower)
+                            if (f8) {
+                                ptx::tma_load_3d_pair(a_dst, &map_a8, bar0, x, row_a, p.ia[k]);
+                                ptx::tma_load_3d_pair(a_dst + kABytes, &map_b8, bar0, x, row_b, p.ib[k]);
+                            } else {
+                                ptx::tma_load_3d_pair(a_dst, &map_a, bar0, x, row_a, p.ia[k]);
+                                ptx::tma_load_3d_pair(a_dst + kABytes, &map_b, bar0, x, row_b, p.ib[k]);
+                            }
                         } else {
                             ptx::mbar_arrive_expect_tx(bar, kStageBytes);
                             ptx::tma_load_3d(a_dst, &map_a, bar, x, row_a, p.ia[k]);
@@ -271,6 +277,36 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // ---------------------------------------------------------------- MMA issuer
             uint32_t it = 0, drains = 0;
             bool ok = true;
+            // One accumulation segment: K blocks [kb0, kb_end) into the accumulator at acc_col.  The
+            // operand format is a compile-time constant of the loop: a per-instruction test of a
+            // run-time flag here slowed every instruction of either format by half.
+            auto issue_segment = [&](auto is_f8, int kb0, int kb_end, uint32_t acc_col) {
+                constexpr bool kF8 = decltype(is_f8)::value;
+                for (int kb = kb0; kb < kb_end; ++kb, ++it) {
+                    const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+                    if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->full[s]), ph, p.status, 3))) break;
+                    ptx::tc_fence_after();
+                    const uint32_t a_addr = tiles_base + s * kStageBytes;
+                    const uint64_t a_desc = ptx::smem_desc_k_sw128(a_addr);
+                    const uint64_t b_desc = ptx::smem_desc_k_sw128(a_addr + kABytes);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // 32 bytes further along K inside the swizzle row (64 E2M1 or 32 E4M3 elements)
+                        const uint32_t acc = (kb > kb0 || j > 0) ? 1u : 0u;
+                        if (kF8)
+                            ptx::mma_f8_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, C::kIdescF8, acc);
+                        else if (kPair)
+                            ptx::mma_mxf4_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
+                                               tmem + kSfaCol, tmem + kSfbCol, acc);
+                        else
+                            ptx::mma_mxf4(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc, tmem + kSfaCol,
+                                          tmem + kSfbCol, acc);
+                    }
+                    // frees the stage in both CTAs of a pair
+                    if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->empty[s]), 3);
+                    else ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));
+                }
+            };
             for (int t = worker, tile_iter = 0; t < num_tiles && ok; t += num_workers, ++tile_iter) {
                 for (int kk = 0; kk < p.r && ok; ++kk) {
                     const bool f8 = kMixed && p.fp8[product_at(kk, tile_iter, p.r)];
@@ -290,30 +326,8 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             break;
                         ptx::tc_fence_after();
                         const int kb_end = min(nkb, (c + 1) * ckb);
-                        for (int kb = c * ckb; kb < kb_end; ++kb, ++it) {
-                            const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
-                            if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->full[s]), ph, p.status, 3))) break;
-                            ptx::tc_fence_after();
-                            const uint32_t a_addr = tiles_base + s * kStageBytes;
-                            const uint64_t a_desc = ptx::smem_desc_k_sw128(a_addr);
-                            const uint64_t b_desc = ptx::smem_desc_k_sw128(a_addr + kABytes);
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                // 64 elements = 32 bytes further along K inside the swizzle row
-                                const uint32_t acc = (kb > c * ckb || j > 0) ? 1u : 0u;
-                                if (f8)
-                                    ptx::mma_f8_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, C::kIdescF8, acc);
-                                else if (kPair)
-                                    ptx::mma_mxf4_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
-                                                       tmem + kSfaCol, tmem + kSfbCol, acc);
-                                else
-                                    ptx::mma_mxf4(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
-                                                  tmem + kSfaCol, tmem + kSfbCol, acc);
-                            }
-                            // frees the stage in both CTAs of a pair
-                            if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->empty[s]), 3);
-                            else ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));
-                        }
+                        if (kMixed && f8) issue_segment(std::true_type{}, c * ckb, kb_end, acc_col);
+                        else issue_segment(std::false_type{}, c * ckb, kb_end, acc_col);
                         if (ok) {
                             if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->acc_full[ab]), 3);
                             else ptx::mma_commit(ptx::smem_u32(&sh->acc_full[ab]));
