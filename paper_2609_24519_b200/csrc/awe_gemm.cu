@@ -14,6 +14,10 @@
 // running sum.  After the last product the sum is shifted by log2 D (Definition 4.1) or reduced
 // mod m (Section 5.3) and written once.
 //
+// Records that mix operand formats (Appendix A: two E4M3 products and one E2M1 product) run in the
+// kMixed instantiation: an E4M3 product streams one-byte elements through the same ring and the
+// same descriptors with tcgen05.mma kind::f8f6f4, and its accumulator holds the product itself.
+//
 // 32-bit wrap-around is deliberate: sum_k l_k P_k is computed modulo 2^32, which equals the
 // true D*C whenever |D*C| < 2^31 (checked on the host), although single terms may exceed it.
 //
