@@ -152,9 +152,12 @@ size_t awe_workspace_bytes(int enc, int modulus, int64_t M, int64_t N, int64_t K
 size_t awe_host_staging_bytes(int enc, int modulus, int64_t M, int64_t N, int64_t K, awe_out_dtype_t out_dt);
 
 /* Encode one operand (Algorithm 1, first two loops): table lookup per value, plane formation,
- * E2M1 packing.  X_dev: R x K integers laid out per `layout` with leading dimension ld (elements).
- * planes_dev: awe_planes_bytes bytes, 256-B aligned.  Any ld and any alignment of X_dev are accepted
- * (16-B aligned X_dev and ld % 16 == 0 take the vectorised path). */
+ * E2M1 packing (E4M3 bytes for the FP8 planes of AWE_ENC_INT8_MIXED_FP8_3).  X_dev: R x K integers
+ * laid out per `layout` with leading dimension ld (elements).  planes_dev: awe_planes_bytes bytes,
+ * 256-B aligned.  Any ld and any alignment of X_dev are accepted (16-B aligned X_dev and
+ * ld % 16 == 0 take the vectorised path); AWE_I4_PACKED needs an even ld (AWE_ERR_INVALID_ARG
+ * otherwise) and vectorises with ld % 32 == 0 (R x K layout) or ld % 4 == 0 (K x R layout).
+ * AWE_ERR_UNSUPPORTED if the encoding has no table for `dt` on this side. */
 awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_side_t side, const void* X_dev,
                         awe_in_dtype_t dt, awe_layout_t layout, int64_t R, int64_t K, int64_t ld,
                         void* planes_dev, void* stream);
@@ -171,7 +174,8 @@ awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, const void* p
 
 /* The whole of Algorithm 1: C = A.B exactly (or C mod m).  A_dev: M x K row-major (ld = K),
  * B_dev: K x N row-major (ld = N), C_dev: M x N row-major (ld = N).  workspace_dev: at least
- * awe_workspace_bytes bytes, 256-B aligned; its contents are overwritten. */
+ * awe_workspace_bytes bytes, 256-B aligned; its contents are overwritten.  A packed 4-bit operand
+ * (AWE_I4_PACKED) needs an even K (as A) or an even N (as B). */
 awe_status_t awe_gemm_exact(awe_handle_t h, const void* A_dev, awe_in_dtype_t a_dt, const void* B_dev,
                             awe_in_dtype_t b_dt, int64_t M, int64_t N, int64_t K, int enc, int modulus,
                             void* C_dev, awe_out_dtype_t out_dt, void* workspace_dev, size_t workspace_bytes,
