@@ -156,7 +156,8 @@ __device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128]
 // kMixed: some products of the record multiply E4M3 planes (their own pair of tensor maps, 128
 // elements per 128-byte K block, kind::f8f6f4 without block scales, accumulator = the product
 // itself); the others are E2M1 products as above.  Pair variant only.
-template <bool kPair, bool kMixed>
+// kGrouped: the reconstruction is a weighted sum of cells whose own sums fit 32 bits (GemmParams::group_*).
+template <bool kPair, bool kMixed, bool kGrouped>
 __global__ void __launch_bounds__(kThreads, 1)
 awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a8, const __grid_constant__ CUtensorMap map_b8,
@@ -358,6 +359,9 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             overlap_bar = ptx::map_to_cta(overlap_bar, 0);
             for (int b = 0; b < 2; ++b) acc_empty_bar[b] = ptx::map_to_cta(acc_empty_bar[b], 0);
         }
+        uint32_t* group_scr = nullptr;
+        if (kGrouped)
+            group_scr = p.group_scratch + ((size_t)blockIdx.x * kEpiWarps + (warp - 2)) * (2 * 128 * 32) + lane * 4;
         EpiMath em = {};
         em.out_mode = p.out_mode;
         em.m = m;
@@ -376,12 +380,14 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             uint32_t sum[128];
 #pragma unroll
             for (int i = 0; i < 128; ++i) sum[i] = 0;
+            int n_parked = 0, parked_scale0 = 0, parked_scale1 = 0, last_scale = 1;
             for (int kk = 0; kk < p.r && ok; ++kk) {
                 const int k = product_at(kk, tile_iter, p.r);
                 int ell = p.ell[k];
                 if (m && ell > m_hi) ell -= m;
                 const bool f8 = kMixed && p.fp8[k];
                 if (kMixed) em.acc_scale = f8 ? 1.0f : p.acc_scale;
+
                 const int nchunks = f8 ? chunks8 : chunks;
                 for (int c = 0; c < nchunks && ok; ++c, ++drains) {
                     const uint32_t ab = drains & 1u;
@@ -404,6 +410,23 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         drain_block<3>(taddr + kAccCol1, sum, em, ell);
                     }
                     release(acc_empty_bar[ab], lane, kPair);
+                }
+                if (kGrouped) {
+                    // a cell of the grouped reconstruction is complete when the next product belongs to
+                    // another one: park its 32-bit sum (one coalesced word per lane and column) and start over
+                    last_scale = p.group_scale[k];
+                    if (ok && kk + 1 < p.r && p.group_id[product_at(kk + 1, tile_iter, p.r)] != p.group_id[k]) {
+                        // 16 bytes (4 columns) per lane and store: a warp writes 512 contiguous bytes
+                        uint4* dst = reinterpret_cast<uint4*>(group_scr) + (size_t)n_parked * 32 * 32;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            dst[i * 32] = make_uint4(sum[4 * i], sum[4 * i + 1], sum[4 * i + 2], sum[4 * i + 3]);
+                            sum[4 * i] = sum[4 * i + 1] = sum[4 * i + 2] = sum[4 * i + 3] = 0;
+                        }
+                        if (n_parked == 0) parked_scale0 = last_scale;
+                        else parked_scale1 = last_scale;
+                        ++n_parked;
+                    }
                 }
             }
             if (!ok) break;
@@ -441,9 +464,30 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 uint8_t* gbase = reinterpret_cast<uint8_t*>(p.C) + (row0 * p.ldc + col0) * 8;
 #pragma unroll
                 for (int blk = 0; blk < 8; ++blk) {  // 16 columns = 128 bytes per row
+                    // parked cells of these 16 columns: all loads are issued before the first use (they come
+                    // from L2; taken one by one between the shared-memory stores they cost a latency each)
+                    uint32_t pk0[16], pk1[16];
+                    if (kGrouped) {
+                        const uint4* src = reinterpret_cast<const uint4*>(group_scr) + (size_t)(blk * 4) * 32;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+                            const uint4 a = n_parked > 0 ? src[j * 32] : z;
+                            const uint4 b = n_parked > 1 ? src[(32 + j) * 32] : z;
+                            pk0[4 * j] = a.x; pk0[4 * j + 1] = a.y; pk0[4 * j + 2] = a.z; pk0[4 * j + 3] = a.w;
+                            pk1[4 * j] = b.x; pk1[4 * j + 1] = b.y; pk1[4 * j + 2] = b.z; pk1[4 * j + 3] = b.w;
+                        }
+                    }
                     auto chunk = [&](int c) {
-                        const long long o0 = (long long)((int)sum[blk * 16 + c * 2] >> p.log2D);
-                        const long long o1 = (long long)((int)sum[blk * 16 + c * 2 + 1] >> p.log2D);
+                        long long o0 = (long long)((int)sum[blk * 16 + c * 2] >> p.log2D);
+                        long long o1 = (long long)((int)sum[blk * 16 + c * 2 + 1] >> p.log2D);
+                        if (kGrouped) {
+                            // weighted sum of this cell and the parked ones
+                            o0 = o0 * last_scale + (long long)((int)pk0[c * 2] >> p.log2D) * parked_scale0 +
+                                 (long long)((int)pk1[c * 2] >> p.log2D) * parked_scale1;
+                            o1 = o1 * last_scale + (long long)((int)pk0[c * 2 + 1] >> p.log2D) * parked_scale0 +
+                                 (long long)((int)pk1[c * 2 + 1] >> p.log2D) * parked_scale1;
+                        }
                         return make_uint4((uint32_t)o0, (uint32_t)(o0 >> 32), (uint32_t)o1, (uint32_t)(o1 >> 32));
                     };
                     store_rows_128b<8>(stage, lane, chunk, gbase + blk * 128, p.ldc * 8, rows_valid,
@@ -495,13 +539,13 @@ bool use_pairs() {
     return v;
 }
 
-template <bool kPair, bool kMixed>
+template <bool kPair, bool kMixed, bool kGrouped = false>
 awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ma8,
                             const CUtensorMap& mb8, GemmParams& p, cudaStream_t st) {
     using C = Cfg<kPair>;
-    bool& attr_set = h->smem_attr_set[kMixed ? 3 : (kPair ? 0 : 1)];
+    bool& attr_set = h->smem_attr_set[kGrouped ? 4 : (kMixed ? 3 : (kPair ? 0 : 1))];
     if (!attr_set) {
-        if (cudaFuncSetAttribute(awe_gemm_kernel<kPair, kMixed>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(awe_gemm_kernel<kPair, kMixed, kGrouped>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)C::kSmemBytes) != cudaSuccess)
             return AWE_ERR_CUDA;
         attr_set = true;
@@ -523,7 +567,7 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair, kMixed>, ma, mb, ma8, mb8, p);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair, kMixed, kGrouped>, ma, mb, ma8, mb8, p);
     if (err != cudaSuccess) {
         if (getenv("AWE_DEBUG")) fprintf(stderr, "awe: GEMM launch failed: %s\n", cudaGetErrorString(err));
         return AWE_ERR_CUDA;
@@ -533,6 +577,7 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
 }
 
 awe_status_t launch_gemm(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
+    if (p.group_scratch) return launch_variant<true, false, true>(h, ma, mb, ma, mb, p, st);
     return use_pairs() ? launch_variant<true, false>(h, ma, mb, ma, mb, p, st)
                        : launch_variant<false, false>(h, ma, mb, ma, mb, p, st);
 }
@@ -580,7 +625,17 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
     const int64_t pitch = plane_pitch_bytes(K);
     // 64-bit running sums are needed when not even one 256-element K block keeps D*C within 32 bits
     static const bool force_wide = [] { const char* e = getenv("AWE_FORCE_WIDE_SUMS"); return e && e[0] == '1'; }();
-    const bool wide = !residue && (force_wide || ((int64_t)1 << 30) / (amax * bmax * ((int64_t)1 << d.log2D)) < 256);
+    bool wide = !residue && (force_wide || ((int64_t)1 << 30) / (amax * bmax * ((int64_t)1 << d.log2D)) < 256);
+    // The 12-product record of Appendix A is a sum over limb-pair cells, 2AB = sum_{k,l} 71^(k+l) T_kl
+    // with T_kl = -7 P + 126 P' + 9 Q.  Every T_kl is even and |T_kl| <= 2 * 120^2 * K (the two-limb
+    // halves a_2k + 9 a_2k+1 stay within 12 + 9 * 12), so each cell fits the 32-bit sums of the fast
+    // kernel: the cells of equal weight form a group whose sum is parked, and the tile's 64-bit result is
+    // the sum of the three group sums (halved) with their weights 1, 71 and 5041.
+    struct Group { int first, count, scale; };
+    static const Group kFp16Groups[3] = {{0, 3, 1}, {3, 6, 71}, {9, 3, 5041}};
+    const bool grouped = wide && !force_wide && enc == AWE_ENC_FP16SIG_AWE12 && out_dt == AWE_C_I64 && use_pairs() &&
+                         h->group_scratch_dev != nullptr;
+    if (grouped) wide = false;
     if (wide && !use_pairs()) return AWE_ERR_UNSUPPORTED;
     // E4M3 planes (mixed-format records) come first in the buffer, with rows twice as long
     int n8a = 0, n8b = 0;
@@ -638,6 +693,21 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
         seg_kblocks = std::max<int64_t>(1, std::min(total_kblocks, seg / 256));
     }
     if (residue) seg_kblocks = total_kblocks;
+    if (grouped) {
+        // 2 cells per group at most: |sum| <= 2 * 2 * 120^2 * K_seg must stay below 2^31
+        seg_kblocks = std::min<int64_t>(total_kblocks, (((int64_t)1 << 31) - 1) / (4 * 120 * 120) / 256);
+        int gi = 0;
+        for (const Group& g : kFp16Groups) {
+            for (int k = g.first; k < g.first + g.count; ++k) {
+                if (d.ell[k] % g.scale) return AWE_ERR_UNSUPPORTED;
+                p.ell[k] = d.ell[k] / g.scale;
+                p.group_id[k] = gi;
+                p.group_scale[k] = g.scale;
+            }
+            ++gi;
+        }
+        p.group_scratch = h->group_scratch_dev;
+    }
     for (int64_t kb0 = 0; kb0 < total_kblocks; kb0 += seg_kblocks) {
         p.kblock0 = (int)kb0;
         p.num_kblocks = (int)std::min(seg_kblocks, total_kblocks - kb0);

@@ -80,3 +80,31 @@ def test_fp16sig_8192_sampled_rows():
     assert b.awe_last_device_status(h) == (0, 0)
     for r in (0, 4097, 8191):
         assert np.array_equal(C[r].cpu().numpy(), mm.matmul_i64_s16(A, B, r, r + 1)[0])
+
+
+def test_long_k_runs_in_several_launches_and_keeps_every_cell_within_32_bits():
+    """K beyond the length over which a cell of the grouped reconstruction fits 32 bits (37,120):
+    the launches add into the 64-bit result; all-extreme inputs (including -2048) make every cell as
+    large as it can get."""
+    M, N, K = 256, 128, 45000
+    rng = np.random.default_rng(77)
+    A = rng.choice(np.array([-2048, 2047], np.int16), (M, K))
+    B = rng.choice(np.array([-2048, 2047], np.int16), (K, N))
+    A[0, :] = -2048
+    B[:, 0] = -2048
+    want = mm.matmul_i64_s16(A, B)
+    assert want[0, 0] == 2048 * 2048 * K
+    assert np.array_equal(_run(A, B, b.C_I64), want)
+
+
+def test_many_tiles_per_worker_both_product_orders():
+    """More tiles than workers: every worker walks the products forwards on one tile and backwards on
+    the next, so the cells are parked in either order."""
+    M, N, K = 2560, 2816, 512
+    A, B = wl.make_inputs(wl.small("t", M, N, K, "int12", "int12", seed=9))
+    got = _run(A, B, b.C_I64)
+    rows = [0, 255, 256, 1279, 2559]
+    want = mm.matmul_i64_s16(A[rows], B)
+    assert np.array_equal(got[rows], want)
+    cols = [0, 255, 256, 2815]
+    assert np.array_equal(got[:, cols], mm.matmul_i64_s16(A, np.ascontiguousarray(B[:, cols])))
