@@ -21,9 +21,9 @@ typedef __int128 i128;
 
 struct ResidueParams {
     int n;
-    int m[kMaxModuli];
-    unsigned int c1[kMaxModuli], c2[kMaxModuli], c3[kMaxModuli];  // 2^14, 2^28, 2^42 mod m
-    unsigned int magic[kMaxModuli];                                // floor((2^32 - 1) / m) + 1
+    // per modulus, as floats: m, 1/m, 2^14, 2^28, 2^42 mod m, and the symmetric range
+    float mf[kMaxModuli], inv_m[kMaxModuli], c1f[kMaxModuli], c2f[kMaxModuli], c3f[kMaxModuli];
+    float lo[kMaxModuli], hi[kMaxModuli];
 };
 
 // |x| < 2^56 as four 14-bit limbs l0..l3: |x| = l0 + l1 2^14 + l2 2^28 + l3 2^42.
@@ -43,14 +43,20 @@ __device__ __forceinline__ Limbs14 split14(long long x) {
     return r;
 }
 
-// x mod m in the symmetric range.  s = l0 + l1 c1 + l2 c2 + l3 c3 is congruent to |x| and stays
-// below 2^23, where the 32-bit multiply-high by ceil(2^32 / m) gives the exact quotient.
-__device__ __forceinline__ int symmetric_residue(const Limbs14& v, int m, unsigned int c1, unsigned int c2,
-                                                 unsigned int c3, unsigned int magic) {
-    const unsigned int s = v.l0 + v.l1 * c1 + v.l2 * c2 + v.l3 * c3;
-    int r = (int)(s - __umulhi(s, magic) * (unsigned int)m);  // in [0, m)
-    if (v.neg && r != 0) r = m - r;
-    return r > (m + 1) / 2 - 1 ? r - m : r;
+// x mod m in the symmetric range, on the FP32 pipe (twice the issue rate of 32-bit integer
+// multiplies).  f holds the signed limbs as floats; s = f0 + f1 c1 + f2 c2 + f3 c3 is an integer below 2^24 in magnitude, hence
+// exact; q = round(s / m) by adding and subtracting 1.5 * 2^23, r = s - q m by one exact FMA, and one
+// correction each way puts r into [-floor(m/2), ceil(m/2) - 1] even if q was off by one.  Returns r
+// as the low byte of (r + 1.5 * 2^23)'s bit pattern, i.e. r in two's complement.
+__device__ __forceinline__ uint32_t symmetric_residue_f(const float (&f)[4], float m, float inv_m, float c1, float c2,
+                                                        float c3, float lo, float hi) {
+    const float magic = 12582912.0f;
+    const float sres = __fmaf_rn(f[3], c3, __fmaf_rn(f[2], c2, __fmaf_rn(f[1], c1, f[0])));
+    const float q = __fadd_rn(__fadd_rn(__fmul_rn(sres, inv_m), magic), -magic);
+    float r = __fmaf_rn(-q, m, sres);
+    r = r > hi ? r - m : r;
+    r = r < lo ? r + m : r;
+    return __float_as_uint(r + magic) & 0xFFu;
 }
 
 // X: `count` 64-bit integers; out[t * count + i] = symmetric residue of X[i] modulo m[t].
@@ -72,16 +78,24 @@ wide_residues_kernel(const long long* __restrict__ X, long long count, const __g
             for (int j = 0; j < 4; ++j)
                 if (i0 + j < count) x[j] = X[i0 + j];
         }
-        Limbs14 v[4];
+        float f[4][4];  // signed 14-bit limbs of the four elements
 #pragma unroll
-        for (int j = 0; j < 4; ++j) v[j] = split14(x[j]);
+        for (int j = 0; j < 4; ++j) {
+            const Limbs14 v = split14(x[j]);
+            const float sgn = v.neg ? -1.0f : 1.0f;
+            f[j][0] = sgn * (float)v.l0;
+            f[j][1] = sgn * (float)v.l1;
+            f[j][2] = sgn * (float)v.l2;
+            f[j][3] = sgn * (float)v.l3;
+        }
         const bool full = (i0 + 4 <= count) && ((count & 3) == 0);
+#pragma unroll 2
         for (int t = 0; t < p.n; ++t) {
-            const int m = p.m[t];
+            const float m = p.mf[t], inv_m = p.inv_m[t], c1 = p.c1f[t], c2 = p.c2f[t], c3 = p.c3f[t];
+            const float lo = p.lo[t], hi = p.hi[t];
             uint32_t word = 0;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                word |= ((uint32_t)symmetric_residue(v[j], m, p.c1[t], p.c2[t], p.c3[t], p.magic[t]) & 0xFFu) << (8 * j);
+            for (int j = 0; j < 4; ++j) word |= symmetric_residue_f(f[j], m, inv_m, c1, c2, c3, lo, hi) << (8 * j);
             int8_t* dst = out + (long long)t * count + i0;
             if (full) {
                 *reinterpret_cast<uint32_t*>(dst) = word;
@@ -107,42 +121,84 @@ struct CrtParams {
 // formed limb by limb (four 64-bit accumulators of 32 x 32-bit products, no carries needed: 22 terms
 // below 2^40 each), the quotient by M (< 2^13) is estimated in double precision, q M is subtracted
 // limb by limb, carries are propagated once, and at most two corrections fix the estimate.
+constexpr int kCrtBatch = 12;
+
+// One element: x in (-M/2, M/2] from the four limb sums a0..a3 of sum_t r_t W_t.
+__device__ __forceinline__ i128 crt_reduce(unsigned long long a0, unsigned long long a1, unsigned long long a2,
+                                           unsigned long long a3, const CrtParams& p, i128 M, i128 half) {
+    const double xd = ((double)a3 * 4294967296.0 + (double)a2) * 18446744073709551616.0 +
+                      (double)a1 * 4294967296.0 + (double)a0;
+    const long long q = (long long)floor(xd / p.M_as_double);
+    // d_k = a_k - q M_k (|d_k| < 2^46), then x - q M = sum_k d_k 2^(32 k) with signed carries
+    long long c = (long long)a0 - q * (long long)p.M[0];
+    const unsigned long long r0 = (unsigned long long)c & 0xFFFFFFFFull;
+    c = (c >> 32) + (long long)a1 - q * (long long)p.M[1];
+    const unsigned long long r1 = (unsigned long long)c & 0xFFFFFFFFull;
+    c = (c >> 32) + (long long)a2 - q * (long long)p.M[2];
+    const unsigned long long r2 = (unsigned long long)c & 0xFFFFFFFFull;
+    c = (c >> 32) + (long long)a3 - q * (long long)p.M[3];  // top limb: signed, |c| < 2^28, so its low 32 bits
+    // placed at bit 96 give the right two's-complement value even when the estimate was one too large
+    i128 x = (i128)(((u128)(unsigned long long)c << 96) | ((u128)r2 << 64) | ((u128)r1 << 32) | (u128)r0);
+    if (x < 0) x += M;
+    if (x >= M) x -= M;
+    if (x > half) x -= M;
+    return x;
+}
+
+// A thread takes two neighbouring elements: one 4-byte load per modulus (a warp reads whole 128-byte
+// lines), all loads of a batch of kCrtBatch moduli in flight together (with one 2-byte load at a time
+// the kernel was bound by load latency), and the two 128-bit results leave as one 32-byte sector.
 __global__ void __launch_bounds__(256)
 wide_crt_kernel(const short* __restrict__ res, long long count, const __grid_constant__ CrtParams p,
                 long long* __restrict__ out) {
     const i128 M = (i128)(((u128)p.M_hi << 64) | p.M_lo);
     const i128 half = (i128)(((u128)p.half_hi << 64) | p.half_lo);
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count;
-         i += (long long)gridDim.x * blockDim.x) {
-        unsigned long long a0 = 0, a1 = 0, a2 = 0, a3 = 0;
-#pragma unroll 2
-        for (int t = 0; t < p.n; ++t) {
-            int r = (int)res[(long long)t * count + i];
-            r += r < 0 ? p.m[t] : 0;
-            const unsigned int ru = (unsigned int)r;
-            a0 += (unsigned long long)ru * p.w[t][0];
-            a1 += (unsigned long long)ru * p.w[t][1];
-            a2 += (unsigned long long)ru * p.w[t][2];
-            a3 += (unsigned long long)ru * p.w[t][3];
+    const long long pairs = (count + 1) / 2;
+    // every modulus' array starts on a 4-byte boundary
+    const bool vec = (count & 1) == 0 && (reinterpret_cast<uintptr_t>(res) & 3) == 0;
+    for (long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x; g < pairs;
+         g += (long long)gridDim.x * blockDim.x) {
+        const long long i = 2 * g;
+        const bool two = i + 1 < count;
+        unsigned long long a[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+        for (int t0 = 0; t0 < p.n; t0 += kCrtBatch) {
+            unsigned int word[kCrtBatch];
+#pragma unroll
+            for (int u = 0; u < kCrtBatch; ++u) {
+                word[u] = 0;
+                if (t0 + u < p.n) {
+                    const short* src = res + (long long)(t0 + u) * count + i;
+                    if (vec) {
+                        word[u] = __ldg(reinterpret_cast<const unsigned int*>(src));
+                    } else {
+                        word[u] = (unsigned short)src[0];
+                        if (two) word[u] |= (unsigned int)(unsigned short)src[1] << 16;
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kCrtBatch; ++u) {
+                if (t0 + u >= p.n) break;
+                const int m = p.m[t0 + u];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    int r = (int)(short)(word[u] >> (16 * e));
+                    r += r < 0 ? m : 0;
+                    const unsigned int ru = (unsigned int)r;
+                    a[e][0] += (unsigned long long)ru * p.w[t0 + u][0];
+                    a[e][1] += (unsigned long long)ru * p.w[t0 + u][1];
+                    a[e][2] += (unsigned long long)ru * p.w[t0 + u][2];
+                    a[e][3] += (unsigned long long)ru * p.w[t0 + u][3];
+                }
+            }
         }
-        const double xd = ((double)a3 * 4294967296.0 + (double)a2) * 18446744073709551616.0 +
-                          (double)a1 * 4294967296.0 + (double)a0;
-        const long long q = (long long)floor(xd / p.M_as_double);
-        // d_k = a_k - q M_k (|d_k| < 2^46), then x - q M = sum_k d_k 2^(32 k) with signed carries
-        long long c = (long long)a0 - q * (long long)p.M[0];
-        const unsigned long long r0 = (unsigned long long)c & 0xFFFFFFFFull;
-        c = (c >> 32) + (long long)a1 - q * (long long)p.M[1];
-        const unsigned long long r1 = (unsigned long long)c & 0xFFFFFFFFull;
-        c = (c >> 32) + (long long)a2 - q * (long long)p.M[2];
-        const unsigned long long r2 = (unsigned long long)c & 0xFFFFFFFFull;
-        c = (c >> 32) + (long long)a3 - q * (long long)p.M[3];  // top limb: signed, |c| < 2^28, so its low 32 bits
-        // placed at bit 96 give the right two's-complement value even when the estimate was one too large
-        i128 x = (i128)(((u128)(unsigned long long)c << 96) | ((u128)r2 << 64) | ((u128)r1 << 32) | (u128)r0);
-        if (x < 0) x += M;
-        if (x >= M) x -= M;
-        if (x > half) x -= M;
-        out[2 * i] = (long long)(unsigned long long)(u128)x;
-        out[2 * i + 1] = (long long)(x >> 64);
+        const i128 x0 = crt_reduce(a[0][0], a[0][1], a[0][2], a[0][3], p, M, half);
+        longlong2* dst = reinterpret_cast<longlong2*>(out + 2 * i);
+        dst[0] = make_longlong2((long long)(unsigned long long)(u128)x0, (long long)(x0 >> 64));
+        if (two) {
+            const i128 x1 = crt_reduce(a[1][0], a[1][1], a[1][2], a[1][3], p, M, half);
+            dst[1] = make_longlong2((long long)(unsigned long long)(u128)x1, (long long)(x1 >> 64));
+        }
     }
 }
 
@@ -263,11 +319,13 @@ static awe_status_t launch_residues(awe_handle_t h, const int64_t* X_dev, int64_
     p.n = n;
     for (int t = 0; t < n; ++t) {
         const unsigned int m = (unsigned int)moduli[t];
-        p.m[t] = (int)m;
-        p.c1[t] = (1u << 14) % m;
-        p.c2[t] = (1u << 28) % m;
-        p.c3[t] = (unsigned int)((1ull << 42) % m);
-        p.magic[t] = 0xFFFFFFFFu / m + 1u;
+        p.mf[t] = (float)m;
+        p.inv_m[t] = 1.0f / (float)m;
+        p.c1f[t] = (float)((1u << 14) % m);
+        p.c2f[t] = (float)((1u << 28) % m);
+        p.c3f[t] = (float)((1ull << 42) % m);
+        p.lo[t] = -(float)(m / 2);
+        p.hi[t] = (float)((m + 1) / 2) - 1.0f;
     }
     const long long groups = (count + 3) / 4;
     const unsigned blocks = (unsigned)std::min<long long>((groups + 255) / 256, (long long)h->sm_count * 16);
@@ -288,7 +346,7 @@ static awe_status_t launch_crt(awe_handle_t h, const int16_t* res_dev, int64_t c
     if ((uintptr_t)res_dev % 2 || (uintptr_t)out_dev % 16) return AWE_ERR_ALIGNMENT;
     CrtParams c = {};
     if (!build_crt_params(moduli, n, &c)) return AWE_ERR_UNSUPPORTED;
-    const unsigned blocks = (unsigned)std::min<long long>((count + 255) / 256, (long long)h->sm_count * 16);
+    const unsigned blocks = (unsigned)std::min<long long>(((count + 1) / 2 + 255) / 256, (long long)h->sm_count * 16);
     wide_crt_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const short*)res_dev, count, c, (long long*)out_dev);
     if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
     h->launches += 1;
