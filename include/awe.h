@@ -121,8 +121,7 @@ typedef struct {
 } awe_encoding_desc;
 
 /* Create / destroy a handle bound to CUDA device `device`.  awe_create makes that device
- * current, allocates the handle's status word, table arena (a few hundred KB) and the parking
- * space of the grouped reconstruction of AWE_ENC_FP16SIG_AWE12 (256 KB per SM, 38 MB), once, and
+ * current, allocates the handle's status word and table arena (a few hundred KB, once) and
  * fails with AWE_ERR_CUDA if there is no usable sm_100 device.  (No counterpart in the paper.) */
 awe_status_t awe_create(awe_handle_t* out, int device);
 awe_status_t awe_destroy(awe_handle_t h);

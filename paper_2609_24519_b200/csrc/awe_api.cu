@@ -24,8 +24,7 @@ extern "C" awe_status_t awe_create(awe_handle_t* out, int device) {
     if (cudaMalloc(&h->status_dev, kStatusWords * sizeof(unsigned int)) != cudaSuccess ||
         cudaMemset(h->status_dev, 0, kStatusWords * sizeof(unsigned int)) != cudaSuccess ||
         cudaMalloc(&h->lut_arena_dev, (size_t)kLutSlots * 256 * sizeof(uint64_t)) != cudaSuccess ||
-        cudaMalloc(&h->lut16_arena_dev, (size_t)kLut16Slots * 4096 * sizeof(uint64_t)) != cudaSuccess ||
-        cudaMalloc(&h->group_scratch_dev, (size_t)h->sm_count * kGroupScratchPerCta) != cudaSuccess) {
+        cudaMalloc(&h->lut16_arena_dev, (size_t)kLut16Slots * 4096 * sizeof(uint64_t)) != cudaSuccess) {
         awe_destroy(h);
         return AWE_ERR_CUDA;
     }
@@ -53,7 +52,6 @@ extern "C" awe_status_t awe_destroy(awe_handle_t h) {
     if (h->status_dev) cudaFree(h->status_dev);
     if (h->lut_arena_dev) cudaFree(h->lut_arena_dev);
     if (h->lut16_arena_dev) cudaFree(h->lut16_arena_dev);
-    if (h->group_scratch_dev) cudaFree(h->group_scratch_dev);
     delete h;
     return AWE_OK;
 }

@@ -359,9 +359,6 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             overlap_bar = ptx::map_to_cta(overlap_bar, 0);
             for (int b = 0; b < 2; ++b) acc_empty_bar[b] = ptx::map_to_cta(acc_empty_bar[b], 0);
         }
-        uint32_t* group_scr = nullptr;
-        if (kGrouped)
-            group_scr = p.group_scratch + ((size_t)blockIdx.x * kEpiWarps + (warp - 2)) * (2 * 128 * 32) + lane * 4;
         EpiMath em = {};
         em.out_mode = p.out_mode;
         em.m = m;
@@ -380,7 +377,27 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             uint32_t sum[128];
 #pragma unroll
             for (int i = 0; i < 128; ++i) sum[i] = 0;
-            int n_parked = 0, parked_scale0 = 0, parked_scale1 = 0, last_scale = 1;
+            // ---- tile write-out.  This thread owns one row and 128 consecutive columns; the warp passes
+            // every 128-byte row piece through its shared-memory staging block so that each store
+            // instruction writes 4 rows x 128 contiguous bytes instead of 32 rows x 16 bytes.
+            const long long row0 = (long long)(tm * C::kCtas + (int)rank) * kTileM + quarter * 32;  // first row of the warp
+            const int col0 = tn * kTileN + half * 128;
+            const int rows_valid = (int)max(0ll, min(32ll, (long long)p.M - row0));
+            // 64-bit output: scale * (sum >> log2D), stored or added to what is there
+            auto write_i64 = [&](long long scale, bool add) {
+                uint8_t* gbase = reinterpret_cast<uint8_t*>(p.C) + (row0 * p.ldc + col0) * 8;
+#pragma unroll
+                for (int blk = 0; blk < 8; ++blk) {  // 16 columns = 128 bytes per row
+                    auto chunk = [&](int c) {
+                        const long long o0 = (long long)((int)sum[blk * 16 + c * 2] >> p.log2D) * scale;
+                        const long long o1 = (long long)((int)sum[blk * 16 + c * 2 + 1] >> p.log2D) * scale;
+                        return make_uint4((uint32_t)o0, (uint32_t)(o0 >> 32), (uint32_t)o1, (uint32_t)(o1 >> 32));
+                    };
+                    store_rows_128b<8>(stage, lane, chunk, gbase + blk * 128, p.ldc * 8, rows_valid,
+                                       (p.N - col0 - blk * 16) * 8, p.vec_store, add);
+                }
+            };
+            int flushed = 0;
             for (int kk = 0; kk < p.r && ok; ++kk) {
                 const int k = product_at(kk, tile_iter, p.r);
                 int ell = p.ell[k];
@@ -412,30 +429,21 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     release(acc_empty_bar[ab], lane, kPair);
                 }
                 if (kGrouped) {
-                    // a cell of the grouped reconstruction is complete when the next product belongs to
-                    // another one: park its 32-bit sum (one coalesced word per lane and column) and start over
-                    last_scale = p.group_scale[k];
-                    if (ok && kk + 1 < p.r && p.group_id[product_at(kk + 1, tile_iter, p.r)] != p.group_id[k]) {
-                        // 16 bytes (4 columns) per lane and store: a warp writes 512 contiguous bytes
-                        uint4* dst = reinterpret_cast<uint4*>(group_scr) + (size_t)n_parked * 32 * 32;
+                    // A group of the grouped reconstruction is complete when the next product belongs to
+                    // another one (or there is none): its 32-bit sum goes out with the group's weight,
+                    // stored by the first group of the tile and added by the later ones, while the MMAs of
+                    // the next products run.
+                    const bool last = kk + 1 == p.r;
+                    if (ok && (last || p.group_id[product_at(kk + 1, tile_iter, p.r)] != p.group_id[k])) {
+                        write_i64(p.group_scale[k], flushed > 0 || p.accumulate != 0);
+                        ++flushed;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            dst[i * 32] = make_uint4(sum[4 * i], sum[4 * i + 1], sum[4 * i + 2], sum[4 * i + 3]);
-                            sum[4 * i] = sum[4 * i + 1] = sum[4 * i + 2] = sum[4 * i + 3] = 0;
-                        }
-                        if (n_parked == 0) parked_scale0 = last_scale;
-                        else parked_scale1 = last_scale;
-                        ++n_parked;
+                        for (int i = 0; i < 128; ++i) sum[i] = 0;
                     }
                 }
             }
             if (!ok) break;
-            // ---- write the tile.  This thread owns one row and 128 consecutive columns; the warp
-            // passes every 128-byte row piece through its shared-memory staging block so that each store
-            // instruction writes 4 rows x 128 contiguous bytes instead of 32 rows x 16 bytes.
-            const long long row0 = (long long)(tm * C::kCtas + (int)rank) * kTileM + quarter * 32;  // first row of the warp
-            const int col0 = tn * kTileN + half * 128;
-            const int rows_valid = (int)max(0ll, min(32ll, (long long)p.M - row0));
+            if (kGrouped) continue;  // everything has been written group by group
             if (m) {
                 // residue sums are floats: one last reduction, then to integers in the symmetric range
 #pragma unroll
@@ -461,38 +469,7 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                                        (p.N - col0 - blk * 32) * 4, p.vec_store, false);
                 }
             } else if (p.out_mode == OUT_I64) {
-                uint8_t* gbase = reinterpret_cast<uint8_t*>(p.C) + (row0 * p.ldc + col0) * 8;
-#pragma unroll
-                for (int blk = 0; blk < 8; ++blk) {  // 16 columns = 128 bytes per row
-                    // parked cells of these 16 columns: all loads are issued before the first use (they come
-                    // from L2; taken one by one between the shared-memory stores they cost a latency each)
-                    uint32_t pk0[16], pk1[16];
-                    if (kGrouped) {
-                        const uint4* src = reinterpret_cast<const uint4*>(group_scr) + (size_t)(blk * 4) * 32;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-                            const uint4 a = n_parked > 0 ? src[j * 32] : z;
-                            const uint4 b = n_parked > 1 ? src[(32 + j) * 32] : z;
-                            pk0[4 * j] = a.x; pk0[4 * j + 1] = a.y; pk0[4 * j + 2] = a.z; pk0[4 * j + 3] = a.w;
-                            pk1[4 * j] = b.x; pk1[4 * j + 1] = b.y; pk1[4 * j + 2] = b.z; pk1[4 * j + 3] = b.w;
-                        }
-                    }
-                    auto chunk = [&](int c) {
-                        long long o0 = (long long)((int)sum[blk * 16 + c * 2] >> p.log2D);
-                        long long o1 = (long long)((int)sum[blk * 16 + c * 2 + 1] >> p.log2D);
-                        if (kGrouped) {
-                            // weighted sum of this cell and the parked ones
-                            o0 = o0 * last_scale + (long long)((int)pk0[c * 2] >> p.log2D) * parked_scale0 +
-                                 (long long)((int)pk1[c * 2] >> p.log2D) * parked_scale1;
-                            o1 = o1 * last_scale + (long long)((int)pk0[c * 2 + 1] >> p.log2D) * parked_scale0 +
-                                 (long long)((int)pk1[c * 2 + 1] >> p.log2D) * parked_scale1;
-                        }
-                        return make_uint4((uint32_t)o0, (uint32_t)(o0 >> 32), (uint32_t)o1, (uint32_t)(o1 >> 32));
-                    };
-                    store_rows_128b<8>(stage, lane, chunk, gbase + blk * 128, p.ldc * 8, rows_valid,
-                                       (p.N - col0 - blk * 16) * 8, p.vec_store, p.accumulate != 0);
-                }
+                write_i64(1, p.accumulate != 0);
             } else {  // OUT_RES_I16
                 uint8_t* gbase = reinterpret_cast<uint8_t*>(p.C) + (row0 * p.ldc + col0) * 2;
 #pragma unroll
@@ -577,7 +554,7 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
 }
 
 awe_status_t launch_gemm(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
-    if (p.group_scratch) return launch_variant<true, false, true>(h, ma, mb, ma, mb, p, st);
+    if (p.grouped) return launch_variant<true, false, true>(h, ma, mb, ma, mb, p, st);
     return use_pairs() ? launch_variant<true, false>(h, ma, mb, ma, mb, p, st)
                        : launch_variant<false, false>(h, ma, mb, ma, mb, p, st);
 }
@@ -629,12 +606,11 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
     // The 12-product record of Appendix A is a sum over limb-pair cells, 2AB = sum_{k,l} 71^(k+l) T_kl
     // with T_kl = -7 P + 126 P' + 9 Q.  Every T_kl is even and |T_kl| <= 2 * 120^2 * K (the two-limb
     // halves a_2k + 9 a_2k+1 stay within 12 + 9 * 12), so each cell fits the 32-bit sums of the fast
-    // kernel: the cells of equal weight form a group whose sum is parked, and the tile's 64-bit result is
-    // the sum of the three group sums (halved) with their weights 1, 71 and 5041.
+    // kernel: the cells of equal weight form a group, and the tile's 64-bit result is the sum of the three
+    // group sums (halved) with their weights 1, 71 and 5041, each added to C when its group is done.
     struct Group { int first, count, scale; };
     static const Group kFp16Groups[3] = {{0, 3, 1}, {3, 6, 71}, {9, 3, 5041}};
-    const bool grouped = wide && !force_wide && enc == AWE_ENC_FP16SIG_AWE12 && out_dt == AWE_C_I64 && use_pairs() &&
-                         h->group_scratch_dev != nullptr;
+    const bool grouped = wide && !force_wide && enc == AWE_ENC_FP16SIG_AWE12 && out_dt == AWE_C_I64 && use_pairs();
     if (grouped) wide = false;
     if (wide && !use_pairs()) return AWE_ERR_UNSUPPORTED;
     // E4M3 planes (mixed-format records) come first in the buffer, with rows twice as long
@@ -706,7 +682,7 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
             }
             ++gi;
         }
-        p.group_scratch = h->group_scratch_dev;
+        p.grouped = 1;
     }
     for (int64_t kb0 = 0; kb0 < total_kblocks; kb0 += seg_kblocks) {
         p.kblock0 = (int)kb0;

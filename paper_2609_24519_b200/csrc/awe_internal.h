@@ -64,7 +64,6 @@ struct awe_ctx {
     unsigned int* status_dev = nullptr;  // [0] = status, [1] = site, [2..5] = clock probe of the last GEMM launch
     uint64_t* lut_arena_dev = nullptr;   // kLutSlots tables of 256 x u64
     uint64_t* lut16_arena_dev = nullptr; // kLut16Slots tables of 4096 x u64 (16-bit inputs)
-    uint32_t* group_scratch_dev = nullptr;  // per-CTA parking space for 32-bit group sums (kGroupScratchPerCta each)
     struct Lut16Slot {
         int enc, side;
     };
@@ -88,8 +87,6 @@ namespace awe {
 constexpr int kLutSlots = 96;
 constexpr int kLut16Slots = 4;
 constexpr int kStatusWords = 8;
-// 8 epilogue warps x 2 parked group sums x 128 columns x 32 lanes x 4 bytes
-constexpr size_t kGroupScratchPerCta = 8 * 2 * 128 * 32 * sizeof(uint32_t);
 // Device pointer of the 256-entry u64 table for (enc, modulus, side, dt); uploads on first use.
 awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_in_dtype_t dt,
                         cudaStream_t stream, const uint64_t** out);

@@ -40,12 +40,11 @@ struct GemmParams {
     float acc_scale;   // accumulator value -> product of doubled integers
     uint32_t sf_word;  // four copies of the UE8M0 scale byte
     // Mixed-format records only: products whose planes are E4M3 bytes (128 elements per K block)
-    // Grouped reconstruction (64-bit output only): products with equal group_id form a cell whose
-    // sum fits 32 bits; the result is sum_g group_scale_g * (cell sum >> log2D).  Unused if
-    // group_scratch is null.  Finished cells of a tile wait in group_scratch (kGroupScratchPerCta
-    // bytes per CTA) until the last one is done.
+    // Grouped reconstruction (64-bit output only): products with equal group_id form a group whose
+    // sum fits 32 bits; the result is sum_g group_scale_g * (group sum >> log2D), each group added to
+    // C as soon as it is complete.
+    int grouped;
     int group_id[AWE_MAX_PRODUCTS], group_scale[AWE_MAX_PRODUCTS];
-    uint32_t* group_scratch;
     int fp8[AWE_MAX_PRODUCTS];
     int kblock0_8, num_kblocks8, chunk_kblocks8;
 };
@@ -113,25 +112,17 @@ __device__ __forceinline__ void store_rows_128b(uint8_t* stage, int lane, ChunkF
     __syncwarp();
     const int c = lane & 7;
     if (add64 && elem == 8 && vec_ok && c * 16 + 16 <= bytes_valid) {
-        // read-modify-write of whole 16-byte pieces: four loads of this lane are issued before the
-        // first store, so their latencies overlap instead of adding up
+        // adding to what is there: reductions at L2 (no value comes back, so no load latency is exposed;
+        // integer addition, and no other CTA touches these addresses, so the result is exact and
+        // deterministic)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            longlong2 old[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int r = (h * 4 + i) * 4 + (lane >> 3);
-                if (r < rows_valid) old[i] = *reinterpret_cast<const longlong2*>(gbase + r * row_pitch + c * 16);
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int r = (h * 4 + i) * 4 + (lane >> 3);
-                const uint4 v = *reinterpret_cast<const uint4*>(stage + r * 128 + ((c ^ (r & 7)) << 4));
-                if (r >= rows_valid) continue;
-                const long long a = (long long)(((unsigned long long)v.y << 32) | v.x) + old[i].x;
-                const long long b = (long long)(((unsigned long long)v.w << 32) | v.z) + old[i].y;
-                *reinterpret_cast<longlong2*>(gbase + r * row_pitch + c * 16) = make_longlong2(a, b);
-            }
+        for (int i = 0; i < 8; ++i) {
+            const int r = i * 4 + (lane >> 3);
+            const uint4 v = *reinterpret_cast<const uint4*>(stage + r * 128 + ((c ^ (r & 7)) << 4));
+            if (r >= rows_valid) continue;
+            unsigned long long* dst = reinterpret_cast<unsigned long long*>(gbase + r * row_pitch + c * 16);
+            atomicAdd(dst, ((unsigned long long)v.y << 32) | v.x);
+            atomicAdd(dst + 1, ((unsigned long long)v.w << 32) | v.z);
         }
         __syncwarp();
         return;
