@@ -29,6 +29,7 @@ def test_static_scratch_entry_matches_awe_gemm_exact_twice_in_a_row():
         (wl.small("na1", 384, 520, 1300, seed=41), b.ENC_INT8_AWE6, b.C_I32, torch.int32, 0, b.I8),
         (wl.small("na2", 200, 260, 700, "residue", "residue", seed=42, modulus=89), b.ENC_MOD_M, b.C_RES_I16,
          torch.int16, 89, b.I8),
+        (wl.small("na3", 300, 260, 900, seed=43), b.ENC_INT8_MIXED_FP8_3, b.C_I32, torch.int32, 0, b.I8),
     ]
     for w, enc, out_dt, tdt, modulus, a_dt in cases:          # two calls in a row share the one array
         A_np, B_np = wl.make_inputs(w)
