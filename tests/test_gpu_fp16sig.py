@@ -99,7 +99,7 @@ def test_long_k_runs_in_several_launches_and_keeps_every_cell_within_32_bits():
 
 def test_many_tiles_per_worker_both_product_orders():
     """More tiles than workers: every worker walks the products forwards on one tile and backwards on
-    the next, so the cells are parked in either order."""
+    the next, so the groups reach C in either order."""
     M, N, K = 2560, 2816, 512
     A, B = wl.make_inputs(wl.small("t", M, N, K, "int12", "int12", seed=9))
     got = _run(A, B, b.C_I64)
