@@ -1,5 +1,6 @@
 // Handle management and the whole-procedure entry points (Algorithm 1 end to end).
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <initializer_list>
 #include <new>
@@ -45,10 +46,12 @@ extern "C" awe_status_t awe_destroy(awe_handle_t h) {
     if (h->copy_out) cudaStreamDestroy(h->copy_out);
     for (cudaEvent_t e : {h->ev_start, h->ev_b, h->ev_done})
         if (e) cudaEventDestroy(e);
-    for (int i = 0; i < awe_ctx::kMaxHostChunks; ++i) {
-        if (h->ev_a[i]) cudaEventDestroy(h->ev_a[i]);
-        if (h->ev_c[i]) cudaEventDestroy(h->ev_c[i]);
-    }
+    for (cudaEvent_t e : h->ev_a)
+        if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->ev_bcol)
+        if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->ev_c)
+        if (e) cudaEventDestroy(e);
     if (h->status_dev) cudaFree(h->status_dev);
     if (h->lut_arena_dev) cudaFree(h->lut_arena_dev);
     if (h->lut16_arena_dev) cudaFree(h->lut16_arena_dev);
@@ -185,51 +188,108 @@ extern "C" awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, 
     const int64_t bmax = std::max(std::abs(d.b_lo), std::abs(d.b_hi));
     if (out_dt == AWE_C_I32 && (__int128)amax * bmax * K >= ((__int128)1 << 31)) return AWE_ERR_RANGE;
 
-    // Rows of A (and of C) are cut into chunks so that the copy of chunk i+1 to the device, the
-    // work on chunk i and the copy of chunk i-1 back to the host overlap (the two copy directions
-    // run on their own streams).  Small problems go through in one piece.
-    int chunks = (int)std::min<int64_t>(awe_ctx::kMaxHostChunks, M / 1024);
+    // The product is cut into blocks -- rows of A and C into up to 16 chunks, columns of B and C into up
+    // to 4 blocks, about 2048 x 2048 each (one wave of tile pairs per launch) -- so that the copies to the
+    // device, the kernels and the copies back overlap (the two copy directions run on their own
+    // streams).  The result is twice the bytes of the operands, so the copy back is the long pole: it
+    // starts after one column block of B and one row chunk of A have arrived.  Small problems go
+    // through in one piece.
+    int chunks = (int)std::min<int64_t>(awe_ctx::kMaxHostChunks, M / 2048);
+    int col_blocks = (int)std::min<int64_t>(awe_ctx::kMaxHostColBlocks, N / 2048);
+    if (chunks < 2) {  // few rows: row chunks of 1024 still overlap the copies, without column blocks
+        chunks = (int)std::min<int64_t>(awe_ctx::kMaxHostChunks, M / 1024);
+        col_blocks = 1;
+    }
     if (chunks < 2) chunks = 1;
+    if (col_blocks < 2) col_blocks = 1;
     if (!h->copy_in) {
         bool ok = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) == cudaSuccess &&
                   cudaEventCreateWithFlags(&h->ev_b, cudaEventDisableTiming) == cudaSuccess &&
                   cudaEventCreateWithFlags(&h->ev_done, cudaEventDisableTiming) == cudaSuccess;
-        for (int i = 0; ok && i < awe_ctx::kMaxHostChunks; ++i)
-            ok = cudaEventCreateWithFlags(&h->ev_a[i], cudaEventDisableTiming) == cudaSuccess &&
-                 cudaEventCreateWithFlags(&h->ev_c[i], cudaEventDisableTiming) == cudaSuccess;
+        for (cudaEvent_t& e : h->ev_a) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+        for (cudaEvent_t& e : h->ev_bcol) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+        for (cudaEvent_t& e : h->ev_c) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
         if (!ok) return AWE_ERR_CUDA;
     }
 #define AWE_CU(x) do { if ((x) != cudaSuccess) return AWE_ERR_CUDA; } while (0)
     const int64_t pitch = plane_pitch_bytes(K);
+    const int64_t units_a = t_planes(d, AWE_SIDE_A), units_b = t_planes(d, AWE_SIDE_B);
     uint8_t* pa = base;
     uint8_t* pb = base + round_up((int64_t)awe_planes_bytes(enc, modulus, AWE_SIDE_A, M, K), 256);
+    const int64_t rows_per_chunk = chunks == 1 ? M : round_up((M + chunks - 1) / chunks, 256);
+    const int64_t cols_per_block = col_blocks == 1 ? N : round_up((N + col_blocks - 1) / col_blocks, 256);
+    const int n_row = (int)((M + rows_per_chunk - 1) / rows_per_chunk);
+    const int n_col = (int)((N + cols_per_block - 1) / cols_per_block);
+    const int64_t nib_b = in_elem_nibbles(b_dt);  // half-bytes per element of B
     AWE_CU(cudaEventRecord(h->ev_start, st));
     AWE_CU(cudaStreamWaitEvent(h->copy_in, h->ev_start, 0));
     AWE_CU(cudaStreamWaitEvent(h->copy_out, h->ev_start, 0));
-    AWE_CU(cudaMemcpyAsync(dB, B_host, (size_t)in_bytes(b_dt, K * N), cudaMemcpyHostToDevice, h->copy_in));
-    AWE_CU(cudaEventRecord(h->ev_b, h->copy_in));
-    AWE_CU(cudaStreamWaitEvent(st, h->ev_b, 0));
-    if ((s = awe_encode(h, enc, modulus, AWE_SIDE_B, dB, b_dt, AWE_ROWMAJOR_KxR, N, K, N, pb, stream)) != AWE_OK) return s;
-    const int64_t rows_per_chunk = chunks == 1 ? M : round_up((M + chunks - 1) / chunks, 256);
-    int c = 0;
-    for (int64_t r0 = 0; r0 < M; r0 += rows_per_chunk, ++c) {
-        const int64_t rows = std::min(rows_per_chunk, M - r0);
-        const uint8_t* a_src = (const uint8_t*)A_host + (size_t)in_bytes(a_dt, r0 * K);
-        uint8_t* a_dst = dA + (size_t)in_bytes(a_dt, r0 * K);
-        uint8_t* pa_c = pa + (size_t)t_planes(d, AWE_SIDE_A) * (size_t)r0 * pitch;  // this chunk's own plane block
-        uint8_t* c_dst = dC + (size_t)r0 * N * elem;
-        AWE_CU(cudaMemcpyAsync(a_dst, a_src, (size_t)in_bytes(a_dt, rows * K), cudaMemcpyHostToDevice, h->copy_in));
-        AWE_CU(cudaEventRecord(h->ev_a[c], h->copy_in));
-        AWE_CU(cudaStreamWaitEvent(st, h->ev_a[c], 0));
-        if ((s = awe_encode(h, enc, modulus, AWE_SIDE_A, a_dst, a_dt, AWE_ROWMAJOR_RxK, rows, K, K, pa_c, stream)) != AWE_OK)
+    // Order of the copies to the device: column block 0 of B, the row chunks of A (the copy back of the
+    // first block column keeps pace with them), then the other column blocks of B.
+    auto upload_b = [&](int j) -> awe_status_t {
+        const int64_t c0 = (int64_t)j * cols_per_block, cols = std::min(cols_per_block, N - c0);
+        if (n_col == 1) {
+            AWE_CU(cudaMemcpyAsync(dB, B_host, (size_t)in_bytes(b_dt, K * N), cudaMemcpyHostToDevice, h->copy_in));
+        } else {
+            AWE_CU(cudaMemcpy2DAsync(dB + c0 * nib_b / 2, (size_t)(N * nib_b / 2), (const uint8_t*)B_host + c0 * nib_b / 2,
+                                     (size_t)(N * nib_b / 2), (size_t)(cols * nib_b / 2), (size_t)K,
+                                     cudaMemcpyHostToDevice, h->copy_in));
+        }
+        AWE_CU(cudaEventRecord(h->ev_bcol[j], h->copy_in));
+        return AWE_OK;
+    };
+    auto upload_a = [&](int i) -> awe_status_t {
+        const int64_t r0 = (int64_t)i * rows_per_chunk, rows = std::min(rows_per_chunk, M - r0);
+        AWE_CU(cudaMemcpyAsync(dA + (size_t)in_bytes(a_dt, r0 * K), (const uint8_t*)A_host + (size_t)in_bytes(a_dt, r0 * K),
+                               (size_t)in_bytes(a_dt, rows * K), cudaMemcpyHostToDevice, h->copy_in));
+        AWE_CU(cudaEventRecord(h->ev_a[i], h->copy_in));
+        return AWE_OK;
+    };
+    if ((s = upload_b(0)) != AWE_OK) return s;
+    for (int i = 0; i < n_row; ++i)
+        if ((s = upload_a(i)) != AWE_OK) return s;
+    for (int j = 1; j < n_col; ++j)
+        if ((s = upload_b(j)) != AWE_OK) return s;
+    for (int j = 0; j < n_col; ++j) {
+        const int64_t c0 = (int64_t)j * cols_per_block, cols = std::min(cols_per_block, N - c0);
+        uint8_t* pb_j = pb + (size_t)units_b * (size_t)c0 * pitch;  // this block's own plane set
+        AWE_CU(cudaStreamWaitEvent(st, h->ev_bcol[j], 0));
+        if ((s = awe_encode(h, enc, modulus, AWE_SIDE_B, dB + c0 * nib_b / 2, b_dt, AWE_ROWMAJOR_KxR, cols, K, N, pb_j,
+                            stream)) != AWE_OK)
             return s;
-        if ((s = awe_gemm_planes(h, enc, modulus, pa_c, pb, rows, N, K, c_dst, out_dt, N, 0, stream)) != AWE_OK) return s;
-        AWE_CU(cudaEventRecord(h->ev_c[c], st));
-        AWE_CU(cudaStreamWaitEvent(h->copy_out, h->ev_c[c], 0));
-        AWE_CU(cudaMemcpyAsync((uint8_t*)C_host + (size_t)r0 * N * elem, c_dst, (size_t)rows * N * elem,
-                               cudaMemcpyDeviceToHost, h->copy_out));
+        for (int i = 0; i < n_row; ++i) {
+            const int64_t r0 = (int64_t)i * rows_per_chunk, rows = std::min(rows_per_chunk, M - r0);
+            uint8_t* pa_i = pa + (size_t)units_a * (size_t)r0 * pitch;
+            if (j == 0) {
+                AWE_CU(cudaStreamWaitEvent(st, h->ev_a[i], 0));
+                if ((s = awe_encode(h, enc, modulus, AWE_SIDE_A, dA + (size_t)in_bytes(a_dt, r0 * K), a_dt, AWE_ROWMAJOR_RxK,
+                                    rows, K, K, pa_i, stream)) != AWE_OK)
+                    return s;
+            }
+            uint8_t* c_blk = dC + ((size_t)r0 * N + c0) * elem;
+            if ((s = awe_gemm_planes(h, enc, modulus, pa_i, pb_j, rows, cols, K, c_blk, out_dt, N, 0, stream)) != AWE_OK)
+                return s;
+            // Copy back: block column 0 goes chunk by chunk, so the first bytes leave as early as possible
+            // (its products keep pace with the arrival of A); a later block column is complete long before
+            // the copy of the previous one ends, and goes back as one two-dimensional copy (every copy
+            // costs a gap of some 15 us on the copy stream).
+            const bool per_chunk = j <= 1 || n_col == 1;
+            if (!per_chunk && i + 1 < n_row) continue;
+            cudaEvent_t done = h->ev_c[j * awe_ctx::kMaxHostChunks + i];
+            AWE_CU(cudaEventRecord(done, st));
+            AWE_CU(cudaStreamWaitEvent(h->copy_out, done, 0));
+            const int64_t rr0 = per_chunk ? r0 : 0, rrows = per_chunk ? rows : M;
+            uint8_t* c_dev = dC + ((size_t)rr0 * N + c0) * elem;
+            uint8_t* c_host = (uint8_t*)C_host + ((size_t)rr0 * N + c0) * elem;
+            if (n_col == 1) {
+                AWE_CU(cudaMemcpyAsync(c_host, c_dev, (size_t)rrows * N * elem, cudaMemcpyDeviceToHost, h->copy_out));
+            } else {
+                AWE_CU(cudaMemcpy2DAsync(c_host, (size_t)N * elem, c_dev, (size_t)N * elem, (size_t)cols * elem,
+                                         (size_t)rrows, cudaMemcpyDeviceToHost, h->copy_out));
+            }
+        }
     }
     AWE_CU(cudaEventRecord(h->ev_done, h->copy_out));
     AWE_CU(cudaStreamWaitEvent(st, h->ev_done, 0));

@@ -76,10 +76,12 @@ struct awe_ctx {
     void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
     // copy engines of the host-buffer entry point: one stream per direction and the events that
     // order them against the caller's stream (created on first use)
-    static constexpr int kMaxHostChunks = 16;
+    static constexpr int kMaxHostChunks = 16;   // row chunks of A and C
+    static constexpr int kMaxHostColBlocks = 4;  // column blocks of B and C
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_done = nullptr;
-    cudaEvent_t ev_a[kMaxHostChunks] = {nullptr}, ev_c[kMaxHostChunks] = {nullptr};
+    cudaEvent_t ev_a[kMaxHostChunks] = {nullptr}, ev_bcol[kMaxHostColBlocks] = {nullptr};
+    cudaEvent_t ev_c[kMaxHostChunks * kMaxHostColBlocks] = {nullptr};
     bool smem_attr_set[5] = {false, false, false, false, false};  // dynamic shared-memory limit raised (per kernel, this device)
 };
 

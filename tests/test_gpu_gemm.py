@@ -275,6 +275,32 @@ def test_host_buffer_entry_point_chunked(enc, out_dt, tdt, modulus, kinds):
     assert np.array_equal(Cp.astype(np.int64), want)
 
 
+@pytest.mark.parametrize("enc,out_dt,tdt,kinds,a_dt", [
+    (b.ENC_INT8_AWE6, b.C_I32, torch.int32, ("int8", "int8"), b.I8),
+    (b.ENC_INT8_MIXED_FP8_3, b.C_I64, torch.int64, ("int8", "int8"), b.I8),
+    (b.ENC_INT4xINT8_AWE4, b.C_I32, torch.int32, ("int4", "int8"), b.I4_IN_I8),
+])
+def test_host_buffer_entry_point_row_chunks_and_column_blocks(enc, out_dt, tdt, kinds, a_dt):
+    """M and N large enough for several row chunks and several column blocks, both ragged: the blocks
+    of C come back through two-dimensional copies and must tile the matrix exactly."""
+    h = gu.handle()
+    w = wl.small("t", 4500, 6400, 300, kinds[0], kinds[1], seed=29)
+    A, B = wl.make_inputs(w)
+    Ah, Bh = torch.from_numpy(A).pin_memory(), torch.from_numpy(B).pin_memory()
+    Ch = torch.full((w.M, w.N), 5, dtype=tdt).pin_memory()
+    nbytes = b.awe_workspace_bytes(enc, 0, w.M, w.N, w.K) + b.awe_host_staging_bytes(enc, 0, w.M, w.N, w.K, out_dt)
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    b.awe_gemm_exact_host(h, Ah, a_dt, Bh, b.I8, w.M, w.N, w.K, enc, 0, Ch, out_dt, scratch)
+    assert b.awe_last_device_status(h) == (0, 0)
+    got = Ch.numpy().astype(np.int64)
+    rows = [0, 2047, 2048, 2303, 4095, 4096, 4499]
+    assert np.array_equal(got[rows], mm.matmul_i64(A[rows], B))
+    cols = [0, 2047, 2048, 4095, 4096, 6143, 6144, 6399]
+    assert np.array_equal(got[:, cols], mm.matmul_i64(A, np.ascontiguousarray(B[:, cols])))
+    # whole matrix against the device-buffer entry point
+    assert np.array_equal(got, gu.gpu_gemm_exact(A, B, enc, out_dt, a_dt=a_dt).astype(np.int64))
+
+
 def test_argument_errors_are_reported_before_any_launch():
     h = gu.handle()
     n0 = b.awe_launch_count(h)
