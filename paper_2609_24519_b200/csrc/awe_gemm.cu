@@ -285,7 +285,7 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // One accumulation segment: K blocks [kb0, kb_end) into the accumulator at acc_col.  The
             // operand format is a compile-time constant of the loop: a per-instruction test of a
             // run-time flag here slowed every instruction of either format by half.
-            auto issue_segment = [&](auto is_f8, int kb0, int kb_end, uint32_t acc_col) {
+            auto issue_segment = [&](auto is_f8, int kb0, int kb_end, uint32_t acc_col, bool carry) {
                 constexpr bool kF8 = decltype(is_f8)::value;
                 for (int kb = kb0; kb < kb_end; ++kb, ++it) {
                     const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
@@ -297,7 +297,7 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         // 32 bytes further along K inside the swizzle row (64 E2M1 or 32 E4M3 elements)
-                        const uint32_t acc = (kb > kb0 || j > 0) ? 1u : 0u;
+                        const uint32_t acc = (carry || kb > kb0 || j > 0) ? 1u : 0u;
                         if (kF8)
                             ptx::mma_f8_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, C::kIdescF8, acc);
                         else if (kPair)
@@ -314,28 +314,38 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             };
             for (int t = worker, tile_iter = 0; t < num_tiles && ok; t += num_workers, ++tile_iter) {
                 for (int kk = 0; kk < p.r && ok; ++kk) {
-                    const bool f8 = kMixed && p.fp8[product_at(kk, tile_iter, p.r)];
+                    const int k = product_at(kk, tile_iter, p.r);
+                    const bool f8 = kMixed && p.fp8[k];
                     const int nkb = f8 ? p.num_kblocks8 : p.num_kblocks;
                     const int ckb = f8 ? p.chunk_kblocks8 : p.chunk_kblocks;
                     const int nchunks = f8 ? chunks8 : chunks;
-                    for (int c = 0; c < nchunks && ok; ++c, ++drains) {
+                    // products of one set (equal coefficient; the host merges only when K is a single
+                    // segment) accumulate into the same accumulator and are drained once
+                    const bool set_first = kk == 0 || p.set_id[product_at(kk - 1, tile_iter, p.r)] != p.set_id[k];
+                    const bool set_last = kk + 1 == p.r || p.set_id[product_at(kk + 1, tile_iter, p.r)] != p.set_id[k];
+                    for (int c = 0; c < nchunks && ok; ++c) {
                         // accumulator (drains & 1): its previous contents (two segments ago) fully drained,
                         // and the columns it shares with the other accumulator already read
                         const uint32_t ab = drains & 1u;
                         const uint32_t acc_col = ab ? kAccCol1 : kAccCol0;
-                        if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->acc_empty[ab]), ((drains >> 1) & 1u) ^ 1u,
-                                                p.status, 2)))
-                            break;
-                        if (drains > 0 &&
-                            !(ok = bounded_wait(sh, ptx::smem_u32(&sh->overlap_free), (drains - 1u) & 1u, p.status, 5)))
-                            break;
-                        ptx::tc_fence_after();
+                        if (set_first) {
+                            if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->acc_empty[ab]), ((drains >> 1) & 1u) ^ 1u,
+                                                    p.status, 2)))
+                                break;
+                            if (drains > 0 && !(ok = bounded_wait(sh, ptx::smem_u32(&sh->overlap_free),
+                                                                  (drains - 1u) & 1u, p.status, 5)))
+                                break;
+                            ptx::tc_fence_after();
+                        }
                         const int kb_end = min(nkb, (c + 1) * ckb);
-                        if (kMixed && f8) issue_segment(std::true_type{}, c * ckb, kb_end, acc_col);
-                        else issue_segment(std::false_type{}, c * ckb, kb_end, acc_col);
-                        if (ok) {
-                            if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->acc_full[ab]), 3);
-                            else ptx::mma_commit(ptx::smem_u32(&sh->acc_full[ab]));
+                        if (kMixed && f8) issue_segment(std::true_type{}, c * ckb, kb_end, acc_col, !set_first);
+                        else issue_segment(std::false_type{}, c * ckb, kb_end, acc_col, !set_first);
+                        if (set_last) {
+                            if (ok) {
+                                if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->acc_full[ab]), 3);
+                                else ptx::mma_commit(ptx::smem_u32(&sh->acc_full[ab]));
+                            }
+                            ++drains;
                         }
                     }
                 }
@@ -405,7 +415,9 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 const bool f8 = kMixed && p.fp8[k];
                 if (kMixed) em.acc_scale = f8 ? 1.0f : p.acc_scale;
 
-                const int nchunks = f8 ? chunks8 : chunks;
+                // the accumulator of a merged set is complete after its last product
+                const bool set_last = kk + 1 == p.r || p.set_id[product_at(kk + 1, tile_iter, p.r)] != p.set_id[k];
+                const int nchunks = set_last ? (f8 ? chunks8 : chunks) : 0;
                 for (int c = 0; c < nchunks && ok; ++c, ++drains) {
                     const uint32_t ab = drains & 1u;
                     ok = bounded_wait(sh, ptx::smem_u32(&sh->acc_full[ab]), (drains >> 1) & 1u, p.status, 4);
@@ -683,6 +695,47 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
             ++gi;
         }
         p.grouped = 1;
+    }
+    // Section 3.4: products with the same coefficient can be accumulated together (n_g of them) before
+    // the accumulator is drained, as long as n_g c_A c_B K stays in the exact range.  Only worth doing
+    // where coefficients repeat (base-13: 9 products in 5 sets; the 12-product record: 9 sets; the
+    // four-product residue schemes: 3 sets) and K is a single segment.
+    for (int k = 0; k < d.r; ++k) p.set_id[k] = k;
+    if (!wide) {
+        auto same = [&](int x, int y) {
+            return p.ell[x] == p.ell[y] && p.fp8[x] == p.fp8[y] && p.group_id[x] == p.group_id[y];
+        };
+        int ord[AWE_MAX_PRODUCTS], set_of[AWE_MAX_PRODUCTS], n = 0, n_sets = 0, n_g = 1;
+        bool used[AWE_MAX_PRODUCTS] = {false};
+        for (int k = 0; k < d.r; ++k) {
+            if (used[k]) continue;
+            int run = 0;
+            for (int j = k; j < d.r; ++j)
+                if (!used[j] && same(k, j)) {
+                    used[j] = true;
+                    set_of[n] = n_sets;
+                    ord[n++] = j;
+                    ++run;
+                }
+            n_g = std::max(n_g, run);
+            ++n_sets;
+        }
+        const int64_t k_launch = std::min(seg_kblocks, total_kblocks) * 256;
+        const int64_t exact_range = residue ? ((int64_t)1 << 22) : ((int64_t)1 << 24);
+        if (n_g > 1 && k_launch <= (int64_t)p.chunk_kblocks * 256 &&
+            (int64_t)n_g * d.c_a * d.c_b * k_launch < exact_range) {
+            GemmParams q = p;
+            for (int k = 0; k < d.r; ++k) {
+                q.ia[k] = p.ia[ord[k]];
+                q.ib[k] = p.ib[ord[k]];
+                q.ell[k] = p.ell[ord[k]];
+                q.fp8[k] = p.fp8[ord[k]];
+                q.group_id[k] = p.group_id[ord[k]];
+                q.group_scale[k] = p.group_scale[ord[k]];
+                q.set_id[k] = set_of[k];
+            }
+            p = q;
+        }
     }
     for (int64_t kb0 = 0; kb0 < total_kblocks; kb0 += seg_kblocks) {
         p.kblock0 = (int)kb0;

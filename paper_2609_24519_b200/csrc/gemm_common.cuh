@@ -43,6 +43,9 @@ struct GemmParams {
     // Grouped reconstruction (64-bit output only): products with equal group_id form a group whose
     // sum fits 32 bits; the result is sum_g group_scale_g * (group sum >> log2D), each group added to
     // C as soon as it is complete.
+    // Section 3.4: products with equal coefficient (and format, and group) share one accumulator; they
+    // carry the same set_id and sit next to each other.  All distinct when nothing is merged.
+    int set_id[AWE_MAX_PRODUCTS];
     int grouped;
     int group_id[AWE_MAX_PRODUCTS], group_scale[AWE_MAX_PRODUCTS];
     int fp8[AWE_MAX_PRODUCTS];

@@ -301,6 +301,36 @@ def test_host_buffer_entry_point_row_chunks_and_column_blocks(enc, out_dt, tdt, 
     assert np.array_equal(got, gu.gpu_gemm_exact(A, B, enc, out_dt, a_dt=a_dt).astype(np.int64))
 
 
+def test_merged_accumulators_stay_exact_at_their_bound():
+    """Section 3.4 with n_g > 1: base-13 has up to three products of equal coefficient, which share one
+    accumulator when 3 * 8 * 8 * K < 2^24.  All-(+8) planes at the largest such K (a multiple of 256)
+    put 16,760,832 into the merged accumulators; one K block further the library no longer merges.
+    The planes are not images of int8 data, so the 32-bit result is compared modulo 2^32."""
+    enc = b.ENC_INT8_BASE13_9
+    d = b.awe_encoding_info(enc)
+    assert (d.c_a, d.c_b, d.r) == (8, 8, 9)
+    coeff = sum(int(d.ell[k]) for k in range(d.r))
+    assert coeff == (1 + 13 + 169) ** 2
+    M, N = 128, 256
+    for K in (87296, 87552):
+        assert (3 * 64 * K < 2 ** 24) == (K == 87296)
+        planes = lambda R: np.full((3, R, gu.pitch_bytes(K)), 0x66, dtype=np.uint8)   # E2M1 code 6 = 4.0 -> 8
+        got = gu.gpu_gemm_planes(planes(M), planes(N), M, N, K, enc, b.C_I32)
+        want = np.int64(64 * K * coeff)
+        assert np.all(got.astype(np.int64) & 0xFFFFFFFF == int(want) & 0xFFFFFFFF)
+
+
+def test_equal_coefficient_products_with_real_inputs_and_long_k():
+    """x = 112 = 8 + 13 * 8 on both sides: the merged pair (a0 b1 + a1 b0) is as large as int8 inputs can
+    make it; K just below and above the merging bound of base-13, and the 12-product record alike."""
+    for K in (87296, 87552):
+        A = np.full((130, K), 112, dtype=np.int8)
+        B = np.full((K, 140), -112, dtype=np.int8)
+        B[:, ::2] = 112
+        want = mm.matmul_i64(A, B)
+        assert np.array_equal(gu.gpu_gemm_exact(A, B, b.ENC_INT8_BASE13_9, b.C_I64), want)
+
+
 def test_argument_errors_are_reported_before_any_launch():
     h = gu.handle()
     n0 = b.awe_launch_count(h)
