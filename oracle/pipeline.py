@@ -92,6 +92,27 @@ def plane_products(s: Scheme, pa: np.ndarray, pb: np.ndarray, k_chunk: Optional[
     return np.stack(out) if out else np.zeros((0, pa.shape[1], pb.shape[1]), np.int64)
 
 
+def merged_plane_products(s: Scheme, pa: np.ndarray, pb: np.ndarray) -> Tuple[np.ndarray, List[int]]:
+    """Third loop of Algorithm 1 with products of equal coefficient sharing an accumulator
+    (Section 3.4, n_g > 1): returns one sum per set and the sets' coefficients, asserting that the sum
+    of |products| of every set stays below 2^24 over the whole reduction (one segment)."""
+    from .schemes import equal_coefficient_sets
+    ia, ib = s.plane_index("A"), s.plane_index("B")
+    out, coeff = [], []
+    for members in equal_coefficient_sets(s):
+        acc = np.zeros((pa.shape[1], pb.shape[1]), dtype=np.int64)
+        worst = np.zeros_like(acc)
+        for k in members:
+            a = pa[ia[k]].astype(np.int64)
+            b = pb[ib[k]].astype(np.int64)
+            acc += a @ b.T
+            worst += np.abs(a) @ np.abs(b).T
+        assert worst.max(initial=0) < (1 << F_ACC), "merged partial sum leaves the exact range"
+        out.append(acc)
+        coeff.append(s.ell[members[0]])
+    return np.stack(out), coeff
+
+
 def reconstruct(s: Scheme, P: np.ndarray) -> np.ndarray:
     """Last step of Algorithm 1: C = (sum_k l_k P_k) / D in Python-width integers
     (int64 suffices for every case the tests run), D an exact shift; residue form:

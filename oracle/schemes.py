@@ -174,6 +174,19 @@ def k_star(c_a: int, c_b: int, n_g: int = 1, F: int = F_ACC) -> int:
     return (1 << F) // (n_g * c_a * c_b)
 
 
+def equal_coefficient_sets(s: "Scheme") -> List[List[int]]:
+    """Products that may share one accumulator (Section 3.4, Algorithm 1's third loop): those with the
+    same reconstruction coefficient, listed by first occurrence.  n_g is the size of the largest set."""
+    sets: Dict[int, List[int]] = {}
+    for k, l in enumerate(s.ell):
+        sets.setdefault(l, []).append(k)
+    return list(sets.values())
+
+
+def n_g(s: "Scheme") -> int:
+    return max(len(g) for g in equal_coefficient_sets(s))
+
+
 def x_carry(L: int) -> int:
     """Contiguous half-width of L base-13 limbs, by the recurrence of Section 3.2."""
     return 4 if L == 1 else 13 * x_carry(L - 1) + 4

@@ -174,3 +174,32 @@ def test_tie_break_is_the_stated_one():
             if all(v in sc.S_SET for v in pv) and a[0] + 29 * a[1] + 37 * a[2] == x:
                 cands.append((max(map(abs, pv)), sum(map(abs, pv)), a))
         assert t[x] == min(cands)[2]
+
+
+def test_equal_coefficient_sets_and_their_accumulation_bound():
+    """Section 3.4: n_g products of equal coefficient share an accumulator and divide K* by n_g."""
+    sets = sc.equal_coefficient_sets(sc.BASE13_9)
+    assert sorted(len(g) for g in sets) == [1, 1, 2, 2, 3] and sc.n_g(sc.BASE13_9) == 3
+    # the anti-diagonals i + j = const of the 3 x 3 limb pairs
+    assert sets == [[0], [1, 3], [2, 4, 6], [5, 7], [8]]
+    assert sc.k_star(8, 8, n_g=3) == (1 << 24) // 192 == 87381
+    assert sc.n_g(sc.AWE6) == sc.n_g(sc.AWE6_ALT) == sc.n_g(sc.AWE4) == 1
+    assert sc.n_g(sc.FP16_M12) == 2 and len(sc.equal_coefficient_sets(sc.FP16_M12)) == 9
+    assert sc.n_g(sc.mod_scheme(157)) == 2 and sc.mod_scheme(157).r == 4      # coefficients (1, w1, w1, w1^2)
+    # merged accumulation reconstructs the same matrix
+    rng = np.random.default_rng(8)
+    A = rng.integers(-128, 128, (9, 40), dtype=np.int8)
+    B = rng.integers(-128, 128, (40, 7), dtype=np.int8)
+    for s in (sc.BASE13_9, sc.AWE6):
+        pa = pl.encode_planes(s, "A", A)
+        pb = pl.encode_planes(s, "B", np.ascontiguousarray(B.T))
+        Pm, coeff = pl.merged_plane_products(s, pa, pb)
+        C = sum(np.int64(c) * P for c, P in zip(coeff, Pm)) >> s.log2D
+        assert np.array_equal(C, A.astype(np.int64) @ B.astype(np.int64))
+    # the bound: all-(+8) planes at K = 87,381 stay inside, one more element does not
+    K = 87381
+    pa = np.full((3, 1, K), 8, dtype=np.int8)
+    pl.merged_plane_products(sc.BASE13_9, pa, pa[:, :, :])
+    big = np.full((3, 1, K + 1), 8, dtype=np.int8)
+    with pytest.raises(AssertionError):
+        pl.merged_plane_products(sc.BASE13_9, big, big)
