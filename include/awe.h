@@ -8,6 +8,9 @@
  *   2. for each product k = 1..r, P_k = plane alpha_k of A times plane beta_k of B on the FP4
  *      tensor cores with FP32 accumulation, the reduction dimension cut into segments short
  *      enough (Section 3.4, K*) that every partial sum is an integer below 2^24 and exact;
+ *      products of equal coefficient share an accumulator where that keeps the sum exact (n_g
+ *      of Section 3.4), and the record of Appendix A that mixes formats runs two of its three
+ *      products on E4M3 planes (FP8 tensor cores, same accumulation rule);
  *   3. C = (sum_k l_k P_k) / D in integers, D a power of two (Definition 4.1), or the same sum
  *      reduced mod m for the residue form (Section 5.3)
  *   (steps 2 and 3: awe_gemm_planes; all three: awe_gemm_exact).
