@@ -71,10 +71,14 @@ typedef enum {
     AWE_ENC_FP16SIG_AWE12 = 8,  /* width-12 integers (FP16 significands with sign, |x| <= 2047; the
                                    table also covers -2048), 12 products, w = v = (1,9,71,639), D = 2
                                    (Appendix A).  16-bit inputs (AWE_I16); 64-bit reconstruction.     */
-    AWE_ENC_INT8_MIXED_FP8_3 = 9 /* INT8xINT8 with 2 FP8 products and 1 FP4 product (Appendix A):
+    AWE_ENC_INT8_MIXED_FP8_3 = 9, /* INT8xINT8 with 2 FP8 products and 1 FP4 product (Appendix A):
                                    x = 13 h + 5 eps, planes h and h + eps stored as E4M3 bytes
                                    (|.| <= 14), eps in S (|eps| <= 8) as E2M1;
                                    xy = 104 hh' + 65 (h+eps)(h'+eps') - 40 eps eps', K* = 85,598.     */
+    AWE_ENC_FP8SIG_3 = 10       /* FP8 (E4M3) significands with sign, |x| <= 15 (the table also covers
+                                   -16), 3 products: the Karatsuba-type step on two limbs (Section 6.1;
+                                   the weights are not printed: w = v = (1,4), planes a0, a1, a0-a1,
+                                   xy = 5 a0b0 + 20 a1b1 - 4 (a0-a1)(b0-b1)).  Inputs AWE_I5_IN_I8.    */
 } awe_encoding_t;
 
 typedef enum {
@@ -83,9 +87,10 @@ typedef enum {
     AWE_T2_IN_I8 = 2, /* one ternary value -1, 0 or +1 per byte; any other byte is read as 0         */
     AWE_I16 = 3,      /* one signed 12-bit value per 16-bit element; only the low 12 bits are read
                          (sign-extended).  Leading dimensions stay in elements.                      */
-    AWE_I4_PACKED = 4 /* two signed 4-bit values per byte: element e of the row-major array sits in
+    AWE_I4_PACKED = 4, /* two signed 4-bit values per byte: element e of the row-major array sits in
                          byte e/2, the even one in the low nibble.  Leading dimensions stay in
                          elements and must be even (every row starts on a byte boundary).            */
+    AWE_I5_IN_I8 = 5  /* one signed 5-bit value per byte; only the low 5 bits are read (sign-extended) */
 } awe_in_dtype_t;
 
 typedef enum {

@@ -230,6 +230,13 @@ INT4X4_3 = Scheme("int4xint4_3", (1, 3), (1, 3), ((1, 0), (0, 1), (1, -1)), ((1,
                   (4, 12, -3))
 
 
+# Section 6.1: an E4M3 significand with sign (|x| <= 15) fits two limbs, so the exact product takes
+# the 3 products of the (2,2) cell.  The weights are not printed; same construction as above with
+# w1 = 4, the weight with the smallest plane values (3) over [-15, 15] (coverage 20).
+FP8SIG_3 = Scheme("fp8sig_3", (1, 4), (1, 4), ((1, 0), (0, 1), (1, -1)), ((1, 0), (0, 1), (1, -1)),
+                  (5, 20, -4))
+
+
 def _fp16_m12() -> Scheme:
     """Appendix A, "FP16xFP16 in 12 products": w = (1, 9, 71, 639),
     2AB = sum_{k,l} 71^(k+l) (-7 P[2k,2l] + 126 P[2k+1,2l+1] + 9 Q[k,l])."""

@@ -23,7 +23,8 @@ ENC_TERNARY_INT8_3 = 6
 ENC_INT4xINT4_3 = 7
 ENC_FP16SIG_AWE12 = 8
 ENC_INT8_MIXED_FP8_3 = 9
-I8, I4_IN_I8, T2_IN_I8, I16, I4_PACKED = 0, 1, 2, 3, 4
+ENC_FP8SIG_3 = 10
+I8, I4_IN_I8, T2_IN_I8, I16, I4_PACKED, I5_IN_I8 = 0, 1, 2, 3, 4, 5
 C_I32, C_I64, C_RES_I16, C_RES_I32 = 0, 1, 2, 3
 SIDE_A, SIDE_B = 0, 1
 ROWMAJOR_RxK, ROWMAJOR_KxR = 0, 1

@@ -493,7 +493,7 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
                                    void* planes_dev, void* stream) {
     if (!h || !X_dev || !planes_dev || R <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
     if (side != AWE_SIDE_A && side != AWE_SIDE_B) return AWE_ERR_INVALID_ARG;
-    if ((int)dt < 0 || (int)dt > 4) return AWE_ERR_INVALID_ARG;
+    if ((int)dt < 0 || (int)dt > 5) return AWE_ERR_INVALID_ARG;
     if (layout != AWE_ROWMAJOR_RxK && layout != AWE_ROWMAJOR_KxR) return AWE_ERR_INVALID_ARG;
     if (dt == AWE_I4_PACKED && (ld & 1)) return AWE_ERR_INVALID_ARG;  // rows start on byte boundaries
     if (ld < (layout == AWE_ROWMAJOR_RxK ? K : R)) return AWE_ERR_INVALID_ARG;

@@ -120,6 +120,24 @@ Scheme make_int4x4() {
     return s;
 }
 
+Scheme make_fp8sig() {
+    // x = a0 + 4 a1 on both sides, planes (a0, a1, a0 - a1):
+    //   xy = (1 + 4) a0 b0 + (16 + 4) a1 b1 - 4 (a0 - a1)(b0 - b1)
+    // w1 = 4 is the weight whose tables need the smallest plane values (3) over [-15, 15]
+    Scheme s;
+    s.p = s.q = 2;
+    s.r = 3;
+    set_vec(s.w, {1, 4});
+    set_vec(s.v, {1, 4});
+    const int pl[3][2] = {{1, 0}, {0, 1}, {1, -1}};
+    for (int k = 0; k < 3; ++k)
+        for (int i = 0; i < 2; ++i) s.alpha[k][i] = s.beta[k][i] = pl[k][i];
+    set_vec(s.ell, {5, 20, -4});
+    s.a_lo = s.b_lo = -16;
+    s.a_hi = s.b_hi = 15;
+    return s;
+}
+
 Scheme make_fp16sig() {
     // A = a0 + 9 a1 + 71 a2 + 639 a3 (same for B); with P_ij = a_i b_j and
     // Q_kl = (a_2k + 2 a_2k+1)(b_2l + 2 b_2l+1):
@@ -339,6 +357,7 @@ awe_in_dtype_t natural_dtype(int enc, awe_side_t side) {
     if (enc == AWE_ENC_INT4xINT8_AWE4 && side == AWE_SIDE_A) return AWE_I4_IN_I8;
     if (enc == AWE_ENC_INT4xINT4_3) return AWE_I4_IN_I8;
     if (enc == AWE_ENC_FP16SIG_AWE12) return AWE_I16;
+    if (enc == AWE_ENC_FP8SIG_3) return AWE_I5_IN_I8;
     if (enc == AWE_ENC_TERNARY_INT8_3 && side == AWE_SIDE_A) return AWE_T2_IN_I8;
     return AWE_I8;
 }
@@ -385,6 +404,10 @@ bool get_scheme(int enc, int modulus, Scheme* out) {
             break;
         case AWE_ENC_INT8_MIXED_FP8_3:
             s = make_mixed_fp8();
+            ok = true;
+            break;
+        case AWE_ENC_FP8SIG_3:
+            s = make_fp8sig();
             ok = true;
             break;
         case AWE_ENC_MOD_M:
@@ -459,6 +482,7 @@ bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, co
     for (int b = 0; b < t.entries; ++b) {
         int x = (int)(int8_t)b;
         if (dt == AWE_I4_IN_I8) x = (int)(int8_t)((b & 0xF) << 4) >> 4;  // low nibble, sign-extended
+        if (dt == AWE_I5_IN_I8) x = (int)(int8_t)((b & 0x1F) << 3) >> 3; // low 5 bits, sign-extended
         if (dt == AWE_T2_IN_I8 && (x < -1 || x > 1)) x = 0;              // not a ternary value
         if (dt == AWE_I16) x = (int)(int16_t)((b & 0xFFF) << 4) >> 4;     // low 12 bits, sign-extended
         int key_x = x;
@@ -522,7 +546,7 @@ extern "C" awe_status_t awe_encoding_info(int enc, int modulus, awe_encoding_des
 
 extern "C" awe_status_t awe_encoding_lut(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt,
                                          int8_t* lut_host) {
-    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (int)dt < 0 || (int)dt > 4)
+    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (int)dt < 0 || (int)dt > 5)
         return AWE_ERR_INVALID_ARG;
     const SideTable* t;
     if (!get_side_table(enc, modulus, side, dt, &t)) return AWE_ERR_UNSUPPORTED;

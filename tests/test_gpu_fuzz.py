@@ -20,6 +20,7 @@ KINDS = [
     ("awe4", b.ENC_INT4xINT8_AWE4, b.I4_IN_I8, (-8, 7), b.I8, (-128, 127)),
     ("int4x4", b.ENC_INT4xINT4_3, b.I4_IN_I8, (-8, 7), b.I4_IN_I8, (-8, 7)),
     ("ternary", b.ENC_TERNARY_INT8_3, b.T2_IN_I8, (-1, 1), b.I8, (-128, 127)),
+    ("fp8sig", b.ENC_FP8SIG_3, b.I5_IN_I8, (-16, 15), b.I5_IN_I8, (-16, 15)),
     ("fp16sig", b.ENC_FP16SIG_AWE12, b.I16, (-2047, 2047), b.I16, (-2047, 2047)),
 ]
 
@@ -36,7 +37,7 @@ def _draw(rng, lo, hi, shape, dtype, style):
     return X.astype(dtype)
 
 
-@pytest.mark.parametrize("case", range(48))
+@pytest.mark.parametrize("case", range(54))
 def test_random_shape_and_values(case):
     rng = np.random.default_rng(1000 + case)
     name, enc, a_dt, (alo, ahi), b_dt, (blo, bhi) = KINDS[case % len(KINDS)]

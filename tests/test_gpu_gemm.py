@@ -107,6 +107,26 @@ def test_int4_x_int4_three_products():
         assert np.array_equal(got, mm.matmul_i64(A, B))
 
 
+def test_fp8_significands_three_products():
+    """E4M3 significands with sign (Section 6.1): |x| <= 15 in a 5-bit container; junk above bit 4 is
+    ignored; planes byte for byte against the oracle."""
+    rng = np.random.default_rng(15)
+    A = rng.integers(-15, 16, (300, 1000), dtype=np.int8)
+    B = rng.integers(-15, 16, (1000, 270), dtype=np.int8)
+    A[0, :] = -16
+    B[:, 0] = -16
+    want = mm.matmul_i64(A, B)
+    got = gu.gpu_gemm_exact(A, B, b.ENC_FP8SIG_3, b.C_I32, a_dt=b.I5_IN_I8, b_dt=b.I5_IN_I8)
+    assert np.array_equal(got.astype(np.int64), want)
+    dirty = ((A.astype(np.uint8) & 0x1F) | 0xA0).astype(np.uint8).view(np.int8)
+    got = gu.gpu_gemm_exact(dirty, B, b.ENC_FP8SIG_3, b.C_I32, a_dt=b.I5_IN_I8, b_dt=b.I5_IN_I8)
+    assert np.array_equal(got.astype(np.int64), want)
+    ref = pl.encode_planes(sc.FP8SIG_3, "A", A, -16, 15)
+    packed = gu.padded_planes(np.stack([pl.pack_e2m1(p) for p in ref]), A.shape[1])
+    for layout in (b.ROWMAJOR_RxK, b.ROWMAJOR_KxR):
+        assert np.array_equal(gu.gpu_encode(b.ENC_FP8SIG_3, 0, b.SIDE_A, A, b.I5_IN_I8, layout), packed)
+
+
 def test_ternary_x_int8():
     """Section 6.2: {0, +-1} x INT8 in 3 products (one limb against the three base-13 limbs)."""
     for (M, N, K) in [(256, 512, 1024), (130, 270, 300), (1, 1, 1)]:

@@ -52,6 +52,11 @@ def test_records_match_the_paper_and_the_oracle(b):
     assert d.r == 3 and list(d.ell)[:3] == list(sc.INT4X4_3.ell) and (d.c_a, d.c_b, d.k_star) == (2, 2, 4194304)
     lut = b.awe_encoding_lut(b.ENC_INT4xINT4_3, 0, b.SIDE_B, b.I4_IN_I8)
     assert np.array_equal(lut[np.arange(-8, 8) & 0xFF], pl.plane_lut(sc.INT4X4_3, "B", -8, 7))
+    d = b.awe_encoding_info(b.ENC_FP8SIG_3)
+    assert d.r == 3 and list(d.ell)[:3] == list(sc.FP8SIG_3.ell) and (d.c_a, d.c_b, d.k_star) == (4, 4, 1048576)
+    lut = b.awe_encoding_lut(b.ENC_FP8SIG_3, 0, b.SIDE_A, b.I5_IN_I8)
+    assert np.array_equal(lut[np.arange(-16, 16) & 0x1F], pl.plane_lut(sc.FP8SIG_3, "A", -16, 15))
+    assert np.array_equal(lut[(np.arange(-16, 16) & 0x1F) | 0xE0], pl.plane_lut(sc.FP8SIG_3, "A", -16, 15))
     d = b.awe_encoding_info(b.ENC_INT8_AWE6)
     assert (d.c_a, d.c_b, d.k_star) == (6, 6, 466033)
     d = b.awe_encoding_info(b.ENC_INT4xINT8_AWE4)

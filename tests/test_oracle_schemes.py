@@ -70,7 +70,8 @@ def test_awe6_scalar_coefficient_relations():
     assert (l["P01"], l["P02"], l["P12"]) == (29, 37, 29 * 37)
 
 
-@pytest.mark.parametrize("s", [sc.AWE6, sc.AWE6_ALT, sc.AWE4, sc.BASE13_9, sc.TERNARY3, sc.INT4X4_3, sc.FP16_M12],
+@pytest.mark.parametrize("s", [sc.AWE6, sc.AWE6_ALT, sc.AWE4, sc.BASE13_9, sc.TERNARY3, sc.INT4X4_3, sc.FP8SIG_3,
+                               sc.FP16_M12],
                          ids=lambda s: s.name)
 def test_matrix_identity(s):
     assert sc.coefficient_identity_holds(s)
@@ -140,6 +141,23 @@ def test_int4_x_int4_in_three_products():
     best = min((max(abs(sc.dot(p, sc.value_table((1, w), s.alpha)[x])) for x in range(-8, 8) for p in s.alpha), w)
                for w in range(2, 8) if sc.coverage(sc.value_table((1, w), s.alpha)) >= 8)
     assert best == (2, 3)
+
+
+def test_fp8_significands_in_three_products():
+    # Section 6.1: an E4M3 significand with sign (|x| <= 15) fits 2 limbs, hence the 3 products of the
+    # (2,2) cell; the weights are this oracle's choice by the same rule as for INT4xINT4
+    s = sc.FP8SIG_3
+    assert s.r == 3 and sc.coefficient_identity_holds(s)
+    _all_pairs(s, list(range(-16, 16)), list(range(-16, 16)))
+    t = sc.value_table(s.w, s.alpha)
+    assert sc.coverage(t) == 20 >= 15
+    assert pl.scheme_constants(s, (-15, 15), (-15, 15)) == {"c_A": 3, "c_B": 3, "K_star": (1 << 24) // 9}
+    assert pl.scheme_constants(s, (-16, 15), (-16, 15)) == {"c_A": 4, "c_B": 4, "K_star": 1048576}
+    best = min((max(abs(sc.dot(p, sc.value_table((1, w), s.alpha)[x])) for x in range(-15, 16) for p in s.alpha), w)
+               for w in range(2, 8) if sc.coverage(sc.value_table((1, w), s.alpha)) >= 15)
+    assert best == (3, 4)
+    # every E4M3 significand: 8 + mantissa (normal numbers), 0..7 (subnormals)
+    assert {8 + m for m in range(8)} | set(range(8)) <= set(range(0, 16))
 
 
 def test_all_ternary_x_int8_pairs():
