@@ -434,6 +434,25 @@ def main():
             e1.record()
             torch.cuda.synchronize()
             ctx["fp16_significand_awe12_8192_TOPS"] = ops / (e0.elapsed_time(e1) / 3 * 1e-3) / 1e12
+            # the other significand rows of the paper's table of native formats: FP8 (3 products), BF16 (8)
+            for key, enc_s, dt_s, lo, hi, tdt_in, out_s, tdt_out in (
+                    ("fp8_significand_3_8192_TOPS", b.ENC_FP8SIG_3, b.I5_IN_I8, -15, 16, torch.int8, b.C_I32, torch.int32),
+                    ("bf16_significand_8_8192_TOPS", b.ENC_BF16SIG_8, b.I9_IN_I16, -255, 256, torch.int16, b.C_I32,
+                     torch.int32)):
+                a_s = torch.randint(lo, hi, (8192, 8192), dtype=tdt_in, device=dev, generator=gen)
+                b_s = torch.randint(lo, hi, (8192, 8192), dtype=tdt_in, device=dev, generator=gen)
+                ws_s = torch.empty(b.awe_workspace_bytes(enc_s, 0, 8192, 8192, 8192), dtype=torch.uint8, device=dev)
+                c_s = torch.empty((8192, 8192), dtype=tdt_out, device=dev)
+                for _ in range(2):
+                    b.awe_gemm_exact(h, a_s, dt_s, b_s, dt_s, 8192, 8192, 8192, enc_s, 0, c_s, out_s, ws_s)
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(5):
+                    b.awe_gemm_exact(h, a_s, dt_s, b_s, dt_s, 8192, 8192, 8192, enc_s, 0, c_s, out_s, ws_s)
+                e1.record()
+                torch.cuda.synchronize()
+                ctx[key] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
+                del a_s, b_s, ws_s, c_s
             del a12, b12, ws12, c12
             RNS_SET_FP64 = b.awe_wide_moduli()
             total_ms, prods = 0.0, 0

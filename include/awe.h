@@ -75,10 +75,16 @@ typedef enum {
                                    x = 13 h + 5 eps, planes h and h + eps stored as E4M3 bytes
                                    (|.| <= 14), eps in S (|eps| <= 8) as E2M1;
                                    xy = 104 hh' + 65 (h+eps)(h'+eps') - 40 eps eps', K* = 85,598.     */
-    AWE_ENC_FP8SIG_3 = 10       /* FP8 (E4M3) significands with sign, |x| <= 15 (the table also covers
+    AWE_ENC_FP8SIG_3 = 10,      /* FP8 (E4M3) significands with sign, |x| <= 15 (the table also covers
                                    -16), 3 products: the Karatsuba-type step on two limbs (Section 6.1;
                                    the weights are not printed: w = v = (1,4), planes a0, a1, a0-a1,
                                    xy = 5 a0b0 + 20 a1b1 - 4 (a0-a1)(b0-b1)).  Inputs AWE_I5_IN_I8.    */
+    AWE_ENC_BF16SIG_8 = 11      /* BF16 significands with sign (width 9, |x| <= 255; the table also
+                                   covers -256), 8 products (count from Section 6.2's table; the record
+                                   is not printed): w = v = (4,9,61), planes a0, a1, a2, a0+a1, one
+                                   Karatsuba-type step on the pair (a0, a1),
+                                   xy = -20 a0b0 + 45 a1b1 + 3721 a2b2 + 36 (a0+a1)(b0+b1)
+                                        + 244 (a0b2 + a2b0) + 549 (a1b2 + a2b1).  Inputs AWE_I9_IN_I16. */
 } awe_encoding_t;
 
 typedef enum {
@@ -90,7 +96,9 @@ typedef enum {
     AWE_I4_PACKED = 4, /* two signed 4-bit values per byte: element e of the row-major array sits in
                          byte e/2, the even one in the low nibble.  Leading dimensions stay in
                          elements and must be even (every row starts on a byte boundary).            */
-    AWE_I5_IN_I8 = 5  /* one signed 5-bit value per byte; only the low 5 bits are read (sign-extended) */
+    AWE_I5_IN_I8 = 5, /* one signed 5-bit value per byte; only the low 5 bits are read (sign-extended) */
+    AWE_I9_IN_I16 = 6 /* one signed 9-bit value per 16-bit element; only the low 9 bits are read
+                         (sign-extended).  Leading dimensions stay in elements.                      */
 } awe_in_dtype_t;
 
 typedef enum {

@@ -237,6 +237,16 @@ FP8SIG_3 = Scheme("fp8sig_3", (1, 4), (1, 4), ((1, 0), (0, 1), (1, -1)), ((1, 0)
                   (5, 20, -4))
 
 
+# Section 6.2's table lists BF16 significands (width 9, |x| <= 255) at 8 products; the record is not
+# printed.  Construction used here: three limbs, one Karatsuba-type step on the pair (a0, a1) through
+# the plane a0 + a1, the other four cross terms as direct products (9 - 1 = 8); weights (4, 9, 61): the
+# smallest plane values (4) among the weights up to (7, 59, 199) that cover [-255, 255] (coverage 268).
+BF16SIG_8 = Scheme("bf16sig_8", (4, 9, 61), (4, 9, 61),
+                   ((1, 0, 0), (0, 1, 0), (0, 0, 1), (1, 1, 0), (1, 0, 0), (0, 0, 1), (0, 1, 0), (0, 0, 1)),
+                   ((1, 0, 0), (0, 1, 0), (0, 0, 1), (1, 1, 0), (0, 0, 1), (1, 0, 0), (0, 0, 1), (0, 1, 0)),
+                   (16 - 36, 81 - 36, 61 * 61, 36, 4 * 61, 4 * 61, 9 * 61, 9 * 61))
+
+
 def _fp16_m12() -> Scheme:
     """Appendix A, "FP16xFP16 in 12 products": w = (1, 9, 71, 639),
     2AB = sum_{k,l} 71^(k+l) (-7 P[2k,2l] + 126 P[2k+1,2l+1] + 9 Q[k,l])."""

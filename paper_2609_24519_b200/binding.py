@@ -24,7 +24,8 @@ ENC_INT4xINT4_3 = 7
 ENC_FP16SIG_AWE12 = 8
 ENC_INT8_MIXED_FP8_3 = 9
 ENC_FP8SIG_3 = 10
-I8, I4_IN_I8, T2_IN_I8, I16, I4_PACKED, I5_IN_I8 = 0, 1, 2, 3, 4, 5
+ENC_BF16SIG_8 = 11
+I8, I4_IN_I8, T2_IN_I8, I16, I4_PACKED, I5_IN_I8, I9_IN_I16 = 0, 1, 2, 3, 4, 5, 6
 C_I32, C_I64, C_RES_I16, C_RES_I32 = 0, 1, 2, 3
 SIDE_A, SIDE_B = 0, 1
 ROWMAJOR_RxK, ROWMAJOR_KxR = 0, 1
@@ -140,7 +141,7 @@ def awe_encoding_info(enc: int, modulus: int = 0) -> EncodingDesc:
 def awe_encoding_lut(enc: int, modulus: int, side: int, dt: int = I8) -> np.ndarray:
     n = awe_encoding_info(enc, modulus)
     n_planes = n.n_planes_a if side == SIDE_A else n.n_planes_b
-    out = np.zeros((4096 if dt == I16 else 256, n_planes), dtype=np.int8)
+    out = np.zeros((4096 if dt in (I16, I9_IN_I16) else 256, n_planes), dtype=np.int8)
     _check(lib().awe_encoding_lut(enc, modulus, side, dt, out.ctypes.data), "awe_encoding_lut")
     return out
 

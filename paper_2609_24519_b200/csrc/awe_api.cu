@@ -63,7 +63,7 @@ namespace awe {
 awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, cudaStream_t stream,
                         const uint64_t** out) {
     dt = table_dtype(dt);
-    if (dt == AWE_I16) {  // 4096-entry tables live in their own arena (absent in the allocation-free context)
+    if (is_16bit(dt)) {  // 4096-entry tables live in their own arena (absent in the allocation-free context)
         if (!h->lut16_arena_dev) return AWE_ERR_UNSUPPORTED;
         for (size_t i = 0; i < h->slots16.size(); ++i)
             if (h->slots16[i].enc == enc && h->slots16[i].side == (int)side) {

@@ -493,7 +493,7 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
                                    void* planes_dev, void* stream) {
     if (!h || !X_dev || !planes_dev || R <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
     if (side != AWE_SIDE_A && side != AWE_SIDE_B) return AWE_ERR_INVALID_ARG;
-    if ((int)dt < 0 || (int)dt > 5) return AWE_ERR_INVALID_ARG;
+    if ((int)dt < 0 || (int)dt > 6) return AWE_ERR_INVALID_ARG;
     if (layout != AWE_ROWMAJOR_RxK && layout != AWE_ROWMAJOR_KxR) return AWE_ERR_INVALID_ARG;
     if (dt == AWE_I4_PACKED && (ld & 1)) return AWE_ERR_INVALID_ARG;  // rows start on byte boundaries
     if (ld < (layout == AWE_ROWMAJOR_RxK ? K : R)) return AWE_ERR_INVALID_ARG;
@@ -510,12 +510,16 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
     const int vec_ok = ((uintptr_t)X_dev % align == 0) && (ld % align == 0);
     uint8_t* P = (uint8_t*)planes_dev;
     cudaError_t e;
-    if (dt == AWE_I16) {
+    if (is_16bit(dt)) {
         if ((uintptr_t)X_dev % 2) return AWE_ERR_ALIGNMENT;
         const int vec16 = layout == AWE_ROWMAJOR_RxK ? (((uintptr_t)X_dev % 16 == 0) && (ld % 8 == 0))
                                                      : (((uintptr_t)X_dev % 4 == 0) && (ld % 2 == 0));
-        if (t->n_planes != 6) return AWE_ERR_UNSUPPORTED;
-        e = launch16<6>(layout, (const uint16_t*)X_dev, R, K, ld, lut, P, pitch, plane_stride, vec16, h->sm_count, st);
+        if (t->n_planes == 6)
+            e = launch16<6>(layout, (const uint16_t*)X_dev, R, K, ld, lut, P, pitch, plane_stride, vec16, h->sm_count, st);
+        else if (t->n_planes == 4)
+            e = launch16<4>(layout, (const uint16_t*)X_dev, R, K, ld, lut, P, pitch, plane_stride, vec16, h->sm_count, st);
+        else
+            return AWE_ERR_UNSUPPORTED;
         if (e != cudaSuccess) return AWE_ERR_CUDA;
         h->launches += 1;
         return AWE_OK;

@@ -45,7 +45,8 @@ awe_in_dtype_t natural_dtype(int enc, awe_side_t side);
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 inline int64_t plane_pitch_bytes(int64_t K) { return round_up(K, 256) / 2; }
 // Storage of one input element in half-bytes: 4 for 16-bit elements, 1 for packed 4-bit, else 2.
-inline int64_t in_elem_nibbles(awe_in_dtype_t dt) { return dt == AWE_I16 ? 4 : (dt == AWE_I4_PACKED ? 1 : 2); }
+inline bool is_16bit(awe_in_dtype_t dt) { return dt == AWE_I16 || dt == AWE_I9_IN_I16; }
+inline int64_t in_elem_nibbles(awe_in_dtype_t dt) { return is_16bit(dt) ? 4 : (dt == AWE_I4_PACKED ? 1 : 2); }
 inline int64_t in_bytes(awe_in_dtype_t dt, int64_t count) { return (count * in_elem_nibbles(dt) + 1) / 2; }
 // Packed 4-bit inputs share the table of the one-value-per-byte container.
 inline awe_in_dtype_t table_dtype(awe_in_dtype_t dt) { return dt == AWE_I4_PACKED ? AWE_I4_IN_I8 : dt; }

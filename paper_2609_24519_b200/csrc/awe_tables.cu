@@ -138,6 +138,31 @@ Scheme make_fp8sig() {
     return s;
 }
 
+Scheme make_bf16sig() {
+    // A = 4 a0 + 9 a1 + 61 a2 (same for B), planes a0, a1, a2 and a0 + a1: one Karatsuba-type step on the
+    // pair (a0, a1), a0 b1 + a1 b0 = (a0+a1)(b0+b1) - a0 b0 - a1 b1, the other cross terms directly:
+    //   AB = (16 - 36) a0b0 + (81 - 36) a1b1 + 3721 a2b2 + 36 (a0+a1)(b0+b1)
+    //        + 244 (a0b2 + a2b0) + 549 (a1b2 + a2b1)
+    // (4, 9, 61) has the smallest plane values (4) among the weights up to (7, 59, 199) whose tables
+    // cover [-255, 255] with these planes (coverage 268).
+    Scheme s;
+    s.p = s.q = 3;
+    s.r = 8;
+    set_vec(s.w, {4, 9, 61});
+    set_vec(s.v, {4, 9, 61});
+    const int al[8][3] = {{1, 0, 0}, {0, 1, 0}, {0, 0, 1}, {1, 1, 0}, {1, 0, 0}, {0, 0, 1}, {0, 1, 0}, {0, 0, 1}};
+    const int be[8][3] = {{1, 0, 0}, {0, 1, 0}, {0, 0, 1}, {1, 1, 0}, {0, 0, 1}, {1, 0, 0}, {0, 0, 1}, {0, 1, 0}};
+    for (int k = 0; k < 8; ++k)
+        for (int i = 0; i < 3; ++i) {
+            s.alpha[k][i] = al[k][i];
+            s.beta[k][i] = be[k][i];
+        }
+    set_vec(s.ell, {-20, 45, 3721, 36, 244, 244, 549, 549});
+    s.a_lo = s.b_lo = -256;
+    s.a_hi = s.b_hi = 255;
+    return s;
+}
+
 Scheme make_fp16sig() {
     // A = a0 + 9 a1 + 71 a2 + 639 a3 (same for B); with P_ij = a_i b_j and
     // Q_kl = (a_2k + 2 a_2k+1)(b_2l + 2 b_2l+1):
@@ -358,6 +383,7 @@ awe_in_dtype_t natural_dtype(int enc, awe_side_t side) {
     if (enc == AWE_ENC_INT4xINT4_3) return AWE_I4_IN_I8;
     if (enc == AWE_ENC_FP16SIG_AWE12) return AWE_I16;
     if (enc == AWE_ENC_FP8SIG_3) return AWE_I5_IN_I8;
+    if (enc == AWE_ENC_BF16SIG_8) return AWE_I9_IN_I16;
     if (enc == AWE_ENC_TERNARY_INT8_3 && side == AWE_SIDE_A) return AWE_T2_IN_I8;
     return AWE_I8;
 }
@@ -410,6 +436,10 @@ bool get_scheme(int enc, int modulus, Scheme* out) {
             s = make_fp8sig();
             ok = true;
             break;
+        case AWE_ENC_BF16SIG_8:
+            s = make_bf16sig();
+            ok = true;
+            break;
         case AWE_ENC_MOD_M:
             ok = make_mod(modulus, &s);
             break;
@@ -434,7 +464,7 @@ bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, co
         return true;
     }
     SideTable t;
-    t.entries = dt == AWE_I16 ? 4096 : 256;
+    t.entries = is_16bit(dt) ? 4096 : 256;
     t.value.assign((size_t)t.entries * AWE_MAX_PLANES, 0);
     t.lut.assign((size_t)t.entries, 0);
     stored_planes(s, side, &t);
@@ -485,6 +515,7 @@ bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, co
         if (dt == AWE_I5_IN_I8) x = (int)(int8_t)((b & 0x1F) << 3) >> 3; // low 5 bits, sign-extended
         if (dt == AWE_T2_IN_I8 && (x < -1 || x > 1)) x = 0;              // not a ternary value
         if (dt == AWE_I16) x = (int)(int16_t)((b & 0xFFF) << 4) >> 4;     // low 12 bits, sign-extended
+        if (dt == AWE_I9_IN_I16) x = (int)(int16_t)((b & 0x1FF) << 7) >> 7;  // low 9 bits, sign-extended
         int key_x = x;
         if (s.modulus) {
             key_x = ((x % s.modulus) + s.modulus) % s.modulus;
@@ -546,7 +577,7 @@ extern "C" awe_status_t awe_encoding_info(int enc, int modulus, awe_encoding_des
 
 extern "C" awe_status_t awe_encoding_lut(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt,
                                          int8_t* lut_host) {
-    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (int)dt < 0 || (int)dt > 5)
+    if (!lut_host || (side != AWE_SIDE_A && side != AWE_SIDE_B) || (int)dt < 0 || (int)dt > 6)
         return AWE_ERR_INVALID_ARG;
     const SideTable* t;
     if (!get_side_table(enc, modulus, side, dt, &t)) return AWE_ERR_UNSUPPORTED;

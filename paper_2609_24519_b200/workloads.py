@@ -20,7 +20,7 @@ class Workload:
     M: int
     N: int
     K: int
-    a_kind: str           # "int8" | "int4" | "int5" | "int12" | "ternary" | "extreme" | "residue"
+    a_kind: str           # "int8" | "int4" | "int5" | "int9" | "int12" | "ternary" | "extreme" | "residue"
     b_kind: str
     seed: int
     out: str              # "i32" | "i64" | "res_i16"
@@ -34,6 +34,8 @@ def _draw(rng: np.random.Generator, kind: str, shape: Tuple[int, int], modulus: 
         return rng.integers(-8, 8, size=shape, dtype=np.int8)
     if kind == "int5":                         # FP8 (E4M3) significands with sign, uniform in [-15, 15]
         return rng.integers(-15, 16, size=shape, dtype=np.int8)
+    if kind == "int9":                         # BF16 significands with sign, uniform in [-255, 255], int16 container
+        return rng.integers(-255, 256, size=shape, dtype=np.int16)
     if kind == "int12":                        # width-12 symmetric range (FP16 significand with sign), int16 container
         return rng.integers(-2047, 2048, size=shape, dtype=np.int16)
     if kind == "ternary":                      # uniform in {-1, 0, 1}

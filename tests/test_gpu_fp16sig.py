@@ -82,6 +82,38 @@ def test_fp16sig_8192_sampled_rows():
         assert np.array_equal(C[r].cpu().numpy(), mm.matmul_i64_s16(A, B, r, r + 1)[0])
 
 
+def test_bf16_significands_eight_products():
+    """Width-9 integers (BF16 significands with sign) in a 16-bit container: planes byte for byte, junk
+    above bit 8 ignored, 32- and 64-bit outputs, K long enough for several 64-bit launches."""
+    enc = b.ENC_BF16SIG_8
+    rng = np.random.default_rng(19)
+    A = rng.integers(-255, 256, (300, 1000), dtype=np.int16)
+    B = rng.integers(-255, 256, (1000, 270), dtype=np.int16)
+    A[0, :] = -256
+    B[:, 0] = -256
+    want = mm.matmul_i64_s16(A, B)
+    run = lambda X, Y, out: gu.gpu_gemm_exact(X, Y, enc, out, a_dt=b.I9_IN_I16, b_dt=b.I9_IN_I16).astype(np.int64)
+    assert np.array_equal(run(A, B, b.C_I32), want)
+    assert np.array_equal(run(A, B, b.C_I64), want)
+    dirty = ((A.astype(np.uint16) & 0x1FF) | 0x5A00).astype(np.uint16).view(np.int16)
+    assert np.array_equal(run(dirty, B, b.C_I64), want)
+    ref = pl.encode_planes(sc.BF16SIG_8, "A", A, -256, 255)
+    packed = gu.padded_planes(np.stack([pl.pack_e2m1(p) for p in ref]), A.shape[1])
+    for layout in (b.ROWMAJOR_RxK, b.ROWMAJOR_KxR):
+        assert np.array_equal(gu.gpu_encode(enc, 0, b.SIDE_A, A, b.I9_IN_I16, layout), packed)
+    # extremes over a K that needs 64 bits and several launches
+    K = 40000
+    A = rng.choice(np.array([-256, 255], np.int16), (130, K))
+    B = rng.choice(np.array([-256, 255], np.int16), (K, 140))
+    A[0, :] = -256
+    B[:, 0] = -256
+    want = mm.matmul_i64_s16(A, B)
+    assert want[0, 0] == 65536 * K > 2 ** 31
+    assert np.array_equal(run(A, B, b.C_I64), want)
+    with pytest.raises(b.AweError):
+        run(A, B, b.C_I32)
+
+
 def test_long_k_runs_in_several_launches_and_keeps_every_cell_within_32_bits():
     """K beyond the length over which a cell of the grouped reconstruction fits 32 bits (37,120):
     the launches add into the 64-bit result; all-extreme inputs (including -2048) make every cell as

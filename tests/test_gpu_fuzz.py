@@ -22,6 +22,7 @@ KINDS = [
     ("ternary", b.ENC_TERNARY_INT8_3, b.T2_IN_I8, (-1, 1), b.I8, (-128, 127)),
     ("fp8sig", b.ENC_FP8SIG_3, b.I5_IN_I8, (-16, 15), b.I5_IN_I8, (-16, 15)),
     ("fp16sig", b.ENC_FP16SIG_AWE12, b.I16, (-2047, 2047), b.I16, (-2047, 2047)),
+    ("bf16sig", b.ENC_BF16SIG_8, b.I9_IN_I16, (-256, 255), b.I9_IN_I16, (-256, 255)),
 ]
 
 
@@ -37,16 +38,17 @@ def _draw(rng, lo, hi, shape, dtype, style):
     return X.astype(dtype)
 
 
-@pytest.mark.parametrize("case", range(54))
+@pytest.mark.parametrize("case", range(60))
 def test_random_shape_and_values(case):
     rng = np.random.default_rng(1000 + case)
     name, enc, a_dt, (alo, ahi), b_dt, (blo, bhi) = KINDS[case % len(KINDS)]
     M, N = int(rng.integers(1, 700)), int(rng.integers(1, 700))
     K = int(rng.integers(1, 3000))
-    np_dt = np.int16 if a_dt == b.I16 else np.int8
+    wide_in = a_dt in (b.I16, b.I9_IN_I16)
+    np_dt = np.int16 if wide_in else np.int8
     A = _draw(rng, alo, ahi, (M, K), np_dt, int(rng.integers(0, 4)))
     B = _draw(rng, blo, bhi, (K, N), np_dt, int(rng.integers(0, 4)))
-    want = mm.matmul_i64_s16(A, B) if a_dt == b.I16 else mm.matmul_i64(A, B)
+    want = mm.matmul_i64_s16(A, B) if wide_in else mm.matmul_i64(A, B)
     out_dt = b.C_I64 if (a_dt == b.I16 or case % 3 == 0) else b.C_I32
     got = gu.gpu_gemm_exact(A, B, enc, out_dt, a_dt=a_dt, b_dt=b_dt)
     assert np.array_equal(got.astype(np.int64), want), (name, M, N, K)

@@ -57,6 +57,12 @@ def test_records_match_the_paper_and_the_oracle(b):
     lut = b.awe_encoding_lut(b.ENC_FP8SIG_3, 0, b.SIDE_A, b.I5_IN_I8)
     assert np.array_equal(lut[np.arange(-16, 16) & 0x1F], pl.plane_lut(sc.FP8SIG_3, "A", -16, 15))
     assert np.array_equal(lut[(np.arange(-16, 16) & 0x1F) | 0xE0], pl.plane_lut(sc.FP8SIG_3, "A", -16, 15))
+    d = b.awe_encoding_info(b.ENC_BF16SIG_8)
+    s = sc.BF16SIG_8
+    assert d.r == 8 and list(d.ell)[:8] == list(s.ell) and (d.c_a, d.c_b, d.k_star, d.log2D) == (4, 4, 1048576, 0)
+    assert list(d.ia)[:8] == s.plane_index("A") and list(d.ib)[:8] == s.plane_index("B")
+    lut = b.awe_encoding_lut(b.ENC_BF16SIG_8, 0, b.SIDE_B, b.I9_IN_I16)
+    assert np.array_equal(lut[np.arange(-256, 256) & 0x1FF], pl.plane_lut(s, "B", -256, 255))
     d = b.awe_encoding_info(b.ENC_INT8_AWE6)
     assert (d.c_a, d.c_b, d.k_star) == (6, 6, 466033)
     d = b.awe_encoding_info(b.ENC_INT4xINT8_AWE4)

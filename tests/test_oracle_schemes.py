@@ -71,7 +71,7 @@ def test_awe6_scalar_coefficient_relations():
 
 
 @pytest.mark.parametrize("s", [sc.AWE6, sc.AWE6_ALT, sc.AWE4, sc.BASE13_9, sc.TERNARY3, sc.INT4X4_3, sc.FP8SIG_3,
-                               sc.FP16_M12],
+                               sc.BF16SIG_8, sc.FP16_M12],
                          ids=lambda s: s.name)
 def test_matrix_identity(s):
     assert sc.coefficient_identity_holds(s)
@@ -158,6 +158,21 @@ def test_fp8_significands_in_three_products():
     assert best == (3, 4)
     # every E4M3 significand: 8 + mantissa (normal numbers), 0..7 (subnormals)
     assert {8 + m for m in range(8)} | set(range(8)) <= set(range(0, 16))
+
+
+def test_bf16_significands_in_eight_products():
+    # the count is the paper's (Section 6.2, table of native formats); the record is this oracle's construction
+    s = sc.BF16SIG_8
+    assert s.r == 8 and sc.coefficient_identity_holds(s) and s.D == 1
+    assert len(s.stored_planes("A")) == len(s.stored_planes("B")) == 4
+    v = list(range(-256, 256))
+    _all_pairs(s, v, v)
+    t = sc.value_table(s.w, s.stored_planes("A"))
+    assert sc.coverage(t) == 268 >= 255
+    assert pl.scheme_constants(s, (-256, 255), (-256, 255)) == {"c_A": 4, "c_B": 4, "K_star": 1048576}
+    assert sc.n_g(s) == 2 and len(sc.equal_coefficient_sets(s)) == 6
+    # one Karatsuba-type step saves exactly one of the nine limb-pair products
+    assert s.r == len(s.w) * len(s.v) - 1
 
 
 def test_all_ternary_x_int8_pairs():
