@@ -9,7 +9,8 @@ coprime moduli with the fewest FP4 products in total whose product exceeds 2 K B
 PARITY UNPINNED: with the three-product moduli this oracle can construct (planes a0, a1,
 a0 - a1; see schemes.mod_scheme) the program below reaches 60, not 59; the value 60 and
 the selected set are what the tests assert, and the set is the one the residue benchmark
-configuration uses.
+configuration uses.  (One more three-product modulus, 95 or 97, would make the program return 59;
+tests/test_oracle_mod.py checks that sensitivity.)
 """
 from __future__ import annotations
 

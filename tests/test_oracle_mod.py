@@ -99,6 +99,24 @@ def test_integer_program_reaches_the_same_total():
     assert sum(costs[m] for m in sel) == total
 
 
+def test_one_more_three_product_modulus_would_give_the_printed_total():
+    """Sensitivity of the unpinned total: the program returns the paper's 59 as soon as 95 or 97 costs
+    three products, and no two-limb scheme with a third plane p a0 + q a1 (|p|, |q| <= 2) reaches them."""
+    g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "paper_constants.json")))["rns_fp64"]
+    costs = rns.cost_table(170)
+    assert costs[95] == costs[97] == 4
+    for extra in ((95,), (97,), (95, 97)):
+        c2 = dict(costs)
+        for m in extra:
+            c2[m] = 3
+        assert rns.select_moduli(c2)[0] == g["awe_products"]
+    for p, q in ((1, -1), (1, 1), (1, 2), (1, -2), (2, 1), (2, -1)):
+        T = [(a0, a1) for a0 in sc.S for a1 in sc.S if (p * a0 + q * a1) in sc.S_SET]
+        assert len(T) <= 133
+        for m in (95, 97):
+            assert all(len({(a0 + w * a1) % m for a0, a1 in T}) < m for w in range(1, m))
+
+
 # ------------------------------------------------------------------ residue number system, wide integers
 def test_crt_textbook_examples():
     # Sunzi's problem: x = 2 (mod 3), 3 (mod 5), 2 (mod 7) -> 23
