@@ -137,7 +137,8 @@ typedef struct {
 } awe_encoding_desc;
 
 /* Create / destroy a handle bound to CUDA device `device`.  awe_create makes that device
- * current, allocates the handle's status word and table arena (a few hundred KB, once) and
+ * current, allocates the handle's status word and table arena (about 1 MB, once: room for the
+ * tables of 512 (encoding, modulus, side, container) combinations, more than the library has) and
  * fails with AWE_ERR_CUDA if there is no usable sm_100 device.  (No counterpart in the paper.) */
 awe_status_t awe_create(awe_handle_t* out, int device);
 awe_status_t awe_destroy(awe_handle_t h);
@@ -183,7 +184,10 @@ awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_side_t side, c
  * C_dev: M x N row-major with leading dimension ldc (elements of the output type), aligned to its
  * element size (16-B aligned rows, i.e. C_dev % 16 == 0 and ldc*sizeof(elem) % 16 == 0, take
  * the vector-store path).  k_chunk = 0 lets the library choose the segment length
- * (<= K* and a multiple of 256); a positive multiple of 256 forces it (testing). */
+ * (<= K* and a multiple of 256); a positive multiple of 256 forces it (testing); a forced length
+ * above K* (above a quarter of K* for the residue form) would break exactness and is AWE_ERR_RANGE.
+ * AWE_C_I32 needs D max|a| max|b| K < 2^31 (the sums are formed before the shift by log2 D),
+ * AWE_ERR_RANGE otherwise. */
 awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, const void* planesA_dev,
                              const void* planesB_dev, int64_t M, int64_t N, int64_t K, void* C_dev,
                              awe_out_dtype_t out_dt, int64_t ldc, int64_t k_chunk, void* stream);
@@ -269,15 +273,19 @@ awe_status_t awe_gemm_exact_wide(awe_handle_t h, const int64_t* A_dev, const int
  *   - AWE_ERR_WORKSPACE if awe_workspace_bytes(enc, modulus, M, N, K) exceeds
  *     AWE_STATIC_WORKSPACE_BYTES; nothing is enqueued then.  Encodings with 16-bit inputs are not
  *     served (AWE_ERR_UNSUPPORTED): their 32 KB tables have no room in the built-in array.
- *   - The first call on a device looks up the array's device address and the device's properties
- *     and clears the status word; the first use of an encoding on a device uploads its tables and
- *     waits for that copy.  Make those first calls before any stream capture.
+ *   - The first call on a device looks up the array's device address and the device's properties,
+ *     clears the status word and (once per process) page-locks a small host mirror of the status words
+ *     in place; the first use of an encoding on a device uploads its tables and waits for that copy
+ *     (room for 96 tables per device).  Make those first calls before any stream capture.
  *   - Every call on a device shares the one array, which keeps the previous call's planes: calls
  *     whose kernels could overlap on the GPU (different streams, or several host threads) race
  *     and must be serialised by the caller.  Nothing in it needs to start at zero except the status
  *     word, which the library clears itself.
- *   - A bounded device-side wait that expired during an earlier call is returned (as
- *     AWE_ERR_TIMEOUT, once) by the first later call that finds `stream` idle. */
+ *   - No call waits for the GPU.  Each call ends by enqueuing, on `stream`, a copy of the status word
+ *     into the host mirror; a bounded device-side wait that expired during an earlier call is
+ *     returned (as AWE_ERR_TIMEOUT, once) by the first later call that finds it there, and that call
+ *     enqueues nothing but the clearing of the word: repeat it to get the product.  While `stream` is
+ *     being captured the status word is neither copied nor looked at. */
 awe_status_t awe_gemm_exact_static(const void* A_dev, awe_in_dtype_t a_dt, const void* B_dev, awe_in_dtype_t b_dt,
                                    int64_t M, int64_t N, int64_t K, int enc, int modulus, void* C_dev,
                                    awe_out_dtype_t out_dt, void* stream);

@@ -22,6 +22,7 @@ extern "C" awe_status_t awe_create(awe_handle_t* out, int device) {
     if (!h) return AWE_ERR_CUDA;
     h->device = device;
     h->sm_count = prop.multiProcessorCount;
+    h->lut_slots = kLutSlots;
     if (cudaMalloc(&h->status_dev, kStatusWords * sizeof(unsigned int)) != cudaSuccess ||
         cudaMemset(h->status_dev, 0, kStatusWords * sizeof(unsigned int)) != cudaSuccess ||
         cudaMalloc(&h->lut_arena_dev, (size_t)kLutSlots * 256 * sizeof(uint64_t)) != cudaSuccess ||
@@ -89,7 +90,7 @@ awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_i
             return AWE_OK;
         }
     }
-    if ((int)h->slots.size() >= kLutSlots) return AWE_ERR_UNSUPPORTED;
+    if ((int)h->slots.size() >= h->lut_slots) return AWE_ERR_UNSUPPORTED;
     const SideTable* t;
     if (!get_side_table(enc, modulus, side, dt, &t)) return AWE_ERR_UNSUPPORTED;
     uint64_t* dst = h->lut_arena_dev + h->slots.size() * 256;
@@ -140,9 +141,12 @@ extern "C" awe_status_t awe_gemm_exact(awe_handle_t h, const void* A_dev, awe_in
     const SideTable* t;
     if (!get_side_table(enc, modulus, AWE_SIDE_A, a_dt, &t) || !get_side_table(enc, modulus, AWE_SIDE_B, b_dt, &t))
         return AWE_ERR_UNSUPPORTED;
-    const int64_t amax = std::max(std::abs(d.a_lo), std::abs(d.a_hi));
-    const int64_t bmax = std::max(std::abs(d.b_lo), std::abs(d.b_hi));
-    if (out_dt == AWE_C_I32 && (__int128)amax * bmax * K >= ((__int128)1 << 31)) return AWE_ERR_RANGE;
+    if (out_dt == AWE_C_I32 && !i32_output_fits(d, K)) return AWE_ERR_RANGE;
+    // both tables are on the device (or the arena is known to be full) before the first launch
+    const uint64_t* lut;
+    if ((s = device_lut(h, enc, modulus, AWE_SIDE_A, a_dt, (cudaStream_t)stream, &lut)) != AWE_OK ||
+        (s = device_lut(h, enc, modulus, AWE_SIDE_B, b_dt, (cudaStream_t)stream, &lut)) != AWE_OK)
+        return s;
 
     uint8_t* pa = (uint8_t*)workspace_dev;
     uint8_t* pb = pa + round_up((int64_t)awe_planes_bytes(enc, modulus, AWE_SIDE_A, M, K), 256);
@@ -184,9 +188,11 @@ extern "C" awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, 
     const SideTable* tbl;
     if (!get_side_table(enc, modulus, AWE_SIDE_A, a_dt, &tbl) || !get_side_table(enc, modulus, AWE_SIDE_B, b_dt, &tbl))
         return AWE_ERR_UNSUPPORTED;
-    const int64_t amax = std::max(std::abs(d.a_lo), std::abs(d.a_hi));
-    const int64_t bmax = std::max(std::abs(d.b_lo), std::abs(d.b_hi));
-    if (out_dt == AWE_C_I32 && (__int128)amax * bmax * K >= ((__int128)1 << 31)) return AWE_ERR_RANGE;
+    if (out_dt == AWE_C_I32 && !i32_output_fits(d, K)) return AWE_ERR_RANGE;
+    const uint64_t* lut;
+    if ((s = device_lut(h, enc, modulus, AWE_SIDE_A, a_dt, st, &lut)) != AWE_OK ||
+        (s = device_lut(h, enc, modulus, AWE_SIDE_B, b_dt, st, &lut)) != AWE_OK)
+        return s;
 
     // The product is cut into blocks -- rows of A and C into up to 16 chunks, columns of B and C into up
     // to 4 blocks, about 2048 x 2048 each (one wave of tile pairs per launch) -- so that the copies to the

@@ -609,12 +609,15 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
     // |C| <= max|a| max|b| K must fit the output type
     const int64_t amax = std::max(std::abs(d.a_lo), std::abs(d.a_hi));
     const int64_t bmax = std::max(std::abs(d.b_lo), std::abs(d.b_hi));
-    if (out_dt == AWE_C_I32 && (__int128)amax * bmax * K >= ((__int128)1 << 31)) return AWE_ERR_RANGE;
+    if (out_dt == AWE_C_I32 && !i32_output_fits(d, K)) return AWE_ERR_RANGE;
+    // A forced segment longer than K* (a quarter of it for the residue form, whose epilogue works below
+    // 2^22) would let FP32 partial sums leave the exact range of Section 3.4.
+    if (k_chunk > (residue ? std::max<int64_t>(256, d.k_star / 4) : std::max<int64_t>(256, d.k_star))) return AWE_ERR_RANGE;
 
     const int64_t pitch = plane_pitch_bytes(K);
     // 64-bit running sums are needed when not even one 256-element K block keeps D*C within 32 bits
     static const bool force_wide = [] { const char* e = getenv("AWE_FORCE_WIDE_SUMS"); return e && e[0] == '1'; }();
-    bool wide = !residue && (force_wide || ((int64_t)1 << 30) / (amax * bmax * ((int64_t)1 << d.log2D)) < 256);
+    bool wide = !residue && (force_wide || needs_wide_sums(d));
     // The 12-product record of Appendix A is a sum over limb-pair cells, 2AB = sum_{k,l} 71^(k+l) T_kl
     // with T_kl = -7 P + 126 P' + 9 Q.  Every T_kl is even and |T_kl| <= 2 * 120^2 * K (the two-limb
     // halves a_2k + 9 a_2k+1 stay within 12 + 9 * 12), so each cell fits the 32-bit sums of the fast

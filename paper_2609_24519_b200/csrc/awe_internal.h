@@ -51,6 +51,22 @@ inline int64_t in_bytes(awe_in_dtype_t dt, int64_t count) { return (count * in_e
 // Packed 4-bit inputs share the table of the one-value-per-byte container.
 inline awe_in_dtype_t table_dtype(awe_in_dtype_t dt) { return dt == AWE_I4_PACKED ? AWE_I4_IN_I8 : dt; }
 // Size of one row of all stored planes of a side, in units of the E2M1 pitch.
+// The epilogue keeps sum_k l_k P_k = D*C modulo 2^32 and shifts by log2 D afterwards (Definition 4.1),
+// so 32-bit running sums need |D*C| <= D max|a| max|b| K below 2^31.  When not even one 256-element
+// K block satisfies that, the products run through the kernel with 64-bit sums instead.
+inline int64_t input_bound(const awe_encoding_desc& d) {
+    const int64_t amax = d.a_lo < 0 && -(int64_t)d.a_lo > d.a_hi ? -(int64_t)d.a_lo : d.a_hi;
+    const int64_t bmax = d.b_lo < 0 && -(int64_t)d.b_lo > d.b_hi ? -(int64_t)d.b_lo : d.b_hi;
+    return amax * bmax;
+}
+inline bool needs_wide_sums(const awe_encoding_desc& d) {
+    return d.modulus == 0 && ((int64_t)1 << 30) / (input_bound(d) << d.log2D) < 256;
+}
+// int32 output: the result itself must fit, and so must D*C wherever the sums are 32 bits wide.
+inline bool i32_output_fits(const awe_encoding_desc& d, int64_t K) {
+    const __int128 c = (__int128)input_bound(d) * K;
+    return (needs_wide_sums(d) ? c : c << d.log2D) < ((__int128)1 << 31);
+}
 inline int plane_units(const int32_t* bits, int n_planes) {
     int u = 0;
     for (int j = 0; j < n_planes; ++j) u += bits[j] / 4;
@@ -63,7 +79,8 @@ struct awe_ctx {
     int device = 0;
     int sm_count = 0;
     unsigned int* status_dev = nullptr;  // [0] = status, [1] = site, [2..5] = clock probe of the last GEMM launch
-    uint64_t* lut_arena_dev = nullptr;   // kLutSlots tables of 256 x u64
+    uint64_t* lut_arena_dev = nullptr;   // lut_slots tables of 256 x u64
+    int lut_slots = 0;                   // capacity of that arena
     uint64_t* lut16_arena_dev = nullptr; // kLut16Slots tables of 4096 x u64 (16-bit inputs)
     struct Lut16Slot {
         int enc, side;
@@ -87,7 +104,11 @@ struct awe_ctx {
 };
 
 namespace awe {
-constexpr int kLutSlots = 96;
+// Table arena of a handle: room for both sides of every modulus 2..169 and of every exact
+// encoding in each input container, so that no table ever has to be evicted.
+constexpr int kLutSlots = 512;
+// The allocation-free context keeps its tables inside the built-in array and has room for fewer.
+constexpr int kStaticLutSlots = 96;
 constexpr int kLut16Slots = 4;
 constexpr int kStatusWords = 8;
 // Device pointer of the 256-entry u64 table for (enc, modulus, side, dt); uploads on first use.

@@ -17,7 +17,7 @@ using namespace awe;
 
 namespace {
 
-constexpr size_t kTableBytes = (size_t)kLutSlots * 256 * sizeof(uint64_t);
+constexpr size_t kTableBytes = (size_t)kStaticLutSlots * 256 * sizeof(uint64_t);
 constexpr size_t kStatusBytes = 256;
 constexpr size_t kScratchBytes = (size_t)AWE_STATIC_WORKSPACE_BYTES + kTableBytes + kStatusBytes;
 
@@ -36,6 +36,18 @@ struct DeviceState {
 DeviceState g_state[kMaxDevices];
 std::mutex g_setup_mu;
 
+// Host mirror of each device's status word.  Every call ends with an asynchronous copy of the word
+// into its device's slot, on the caller's stream, and the next call only looks at the slot: no call
+// ever waits for the GPU to learn about an earlier one.  The slots are ordinary library memory,
+// page-locked in place at the first set-up (nothing is allocated) so that those copies really are
+// asynchronous; if the lock is refused the mirror is not used and expired waits go unreported.
+struct alignas(64) StatusSlot {
+    volatile unsigned int word[2];  // status, site
+    unsigned int pad[14];
+};
+alignas(4096) StatusSlot g_status_mirror[kMaxDevices];
+bool g_mirror_tried = false, g_mirror_locked = false;
+
 // One-time set-up for the current device.  Not allocating, but it does query the device and
 // resolves the symbol, so it belongs before any stream capture.
 awe_status_t setup_device(int device, cudaStream_t stream, DeviceState** out) {
@@ -53,12 +65,19 @@ awe_status_t setup_device(int device, cudaStream_t stream, DeviceState** out) {
         s.ctx.device = device;
         s.ctx.sm_count = sms;
         s.ctx.lut_arena_dev = (uint64_t*)(s.base + AWE_STATIC_WORKSPACE_BYTES);
+        s.ctx.lut_slots = kStaticLutSlots;
         s.ctx.status_dev = (unsigned int*)(s.base + AWE_STATIC_WORKSPACE_BYTES + kTableBytes);
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &s.ctx.encode_tiled, cudaEnableDefault, &q) !=
                 cudaSuccess ||
             q != cudaDriverEntryPointSuccess || !s.ctx.encode_tiled)
             return AWE_ERR_CUDA;
+        if (!g_mirror_tried) {
+            g_mirror_tried = true;
+            g_mirror_locked =
+                cudaHostRegister(g_status_mirror, sizeof(g_status_mirror), cudaHostRegisterPortable) == cudaSuccess;
+            if (!g_mirror_locked) cudaGetLastError();  // the refusal is not this call's error
+        }
         // The array keeps whatever an earlier process image or call left: the status word must start at zero.
         if (cudaMemsetAsync(s.ctx.status_dev, 0, kStatusBytes, stream) != cudaSuccess) return AWE_ERR_CUDA;
         s.ready = true;
@@ -82,18 +101,31 @@ extern "C" awe_status_t awe_gemm_exact_static(const void* A_dev, awe_in_dtype_t 
     DeviceState* s = nullptr;
     awe_status_t rc = setup_device(device, st, &s);
     if (rc != AWE_OK) return rc;
-    // A wait that gave up inside an earlier call's kernels is reported by the first later call that
-    // finds the stream idle (checking must not make this call wait for earlier work).
-    if (cudaStreamQuery(st) == cudaSuccess) {
-        unsigned int w[2] = {0, 0};
-        if (cudaMemcpy(w, s->ctx.status_dev, sizeof(w), cudaMemcpyDeviceToHost) != cudaSuccess) return AWE_ERR_CUDA;
-        if (w[0] != 0) {
-            if (cudaMemsetAsync(s->ctx.status_dev, 0, sizeof(w), st) != cudaSuccess) return AWE_ERR_CUDA;
-            return (awe_status_t)w[0];
+    // While `stream` is being captured nothing may be read back or compared on the host: the status
+    // word is left alone and only the kernels are recorded.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) return AWE_ERR_CUDA;
+    const bool report = g_mirror_locked && cap == cudaStreamCaptureStatusNone;
+    // A wait that gave up inside an earlier call's kernels shows up in the host mirror once that
+    // call's trailing copy has run; the call that sees it clears the word, returns the status and does
+    // no other work.
+    if (report) {
+        StatusSlot& slot = g_status_mirror[device];
+        const unsigned int seen = slot.word[0];
+        if (seen != 0) {
+            slot.word[0] = 0;
+            slot.word[1] = 0;
+            if (cudaMemsetAsync(s->ctx.status_dev, 0, 2 * sizeof(unsigned int), st) != cudaSuccess) return AWE_ERR_CUDA;
+            return (awe_status_t)seen;
         }
     }
     // Planes are rewritten in full (padding included) by the encode kernels, so nothing else in the
     // array needs clearing between calls.
-    return awe_gemm_exact(&s->ctx, A_dev, a_dt, B_dev, b_dt, M, N, K, enc, modulus, C_dev, out_dt, s->base,
-                          (size_t)AWE_STATIC_WORKSPACE_BYTES, stream);
+    rc = awe_gemm_exact(&s->ctx, A_dev, a_dt, B_dev, b_dt, M, N, K, enc, modulus, C_dev, out_dt, s->base,
+                        (size_t)AWE_STATIC_WORKSPACE_BYTES, stream);
+    if (rc == AWE_OK && report &&
+        cudaMemcpyAsync((void*)g_status_mirror[device].word, s->ctx.status_dev, 2 * sizeof(unsigned int),
+                        cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return AWE_ERR_CUDA;
+    return rc;
 }

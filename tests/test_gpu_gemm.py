@@ -351,6 +351,26 @@ def test_equal_coefficient_products_with_real_inputs_and_long_k():
         assert np.array_equal(gu.gpu_gemm_exact(A, B, b.ENC_INT8_BASE13_9, b.C_I64), want)
 
 
+def test_int32_output_next_to_the_range_limit_of_the_record_with_D_2():
+    """INT4 x INT8 in 4 products has D = 2 (Appendix A): the 32-bit sums hold 2 C, so int32 output is
+    served while 2 * 8 * 128 * K < 2^31.  K = 2^20 - 256 with the extreme inputs (C = 2^30 - 2^18) is the
+    largest served multiple of 256 and must be exact; K = 2^20 is refused."""
+    K = 2 ** 20 - 256
+    A = np.full((8, K), -8, dtype=np.int8)
+    B = np.full((K, 24), -128, dtype=np.int8)
+    B[:, 1::2] = 127
+    got = gu.gpu_gemm_exact(A, B, b.ENC_INT4xINT8_AWE4, b.C_I32, a_dt=b.I4_IN_I8)
+    want = mm.matmul_i64(A, B)
+    assert want.max() == 2 ** 30 - 2 ** 18 and np.array_equal(got, want)
+    h = gu.handle()
+    x = torch.zeros(16, dtype=torch.int8, device="cuda")
+    with pytest.raises(b.AweError) as e:
+        b.awe_gemm_exact(h, x, b.I4_IN_I8, x, b.I8, 8, 24, 2 ** 20, b.ENC_INT4xINT8_AWE4, 0, x.view(torch.int32), b.C_I32,
+                         torch.empty(b.awe_workspace_bytes(b.ENC_INT4xINT8_AWE4, 0, 8, 24, 2 ** 20), dtype=torch.uint8,
+                                     device="cuda"))
+    assert e.value.status == 5
+
+
 def test_argument_errors_are_reported_before_any_launch():
     h = gu.handle()
     n0 = b.awe_launch_count(h)

@@ -123,3 +123,32 @@ def test_header_is_plain_c():
     r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-fsyntax-only", "-I", os.path.join(ROOT, "include"),
                         "-x", "c", "-"], input=src, capture_output=True, text=True)
     assert r.returncode == 0, r.stderr
+
+
+def test_range_errors_are_returned_before_any_device_work(b):
+    """Definition 4.1's denominator D enters the 32-bit range check, and a forced accumulation
+    segment may not exceed K* (Section 3.4).  Both rejections happen on the host before the handle
+    or any pointer is touched, so a placeholder handle and placeholder addresses reach them."""
+    import ctypes
+    L = b.lib()
+    fake = ctypes.c_void_p(0x10000)          # never dereferenced: the calls return first
+    ptr = ctypes.c_void_p(0x20000)
+
+    def planes(enc, K, out_dt, k_chunk=0, modulus=0):
+        return L.awe_gemm_planes(fake, enc, modulus, ptr, ptr, 256, 256, K, ptr, out_dt, 256, k_chunk, None)
+
+    RANGE = 5
+    # INT4 x INT8 in 4 products has D = 2: |2 C| <= 2 * 8 * 128 * K must stay below 2^31
+    assert planes(b.ENC_INT4xINT8_AWE4, 2 ** 20, b.C_I32) == RANGE
+    assert planes(b.ENC_INT4xINT8_AWE4, 2 ** 21 - 256, b.C_I32) == RANGE
+    # INT8 x INT8 (D = 1): |C| <= 128 * 128 * K
+    assert planes(b.ENC_INT8_AWE6, 2 ** 17, b.C_I32) == RANGE
+    # forced segments beyond K* = 466,033 (6-product record) and beyond K*/4 for a residue record
+    d = b.awe_encoding_info(b.ENC_INT8_AWE6)
+    assert planes(b.ENC_INT8_AWE6, 8192, b.C_I32, k_chunk=(d.k_star // 256 + 1) * 256) == RANGE
+    dm = b.awe_encoding_info(b.ENC_MOD_M, 89)
+    assert planes(b.ENC_MOD_M, 8192, b.C_RES_I16, k_chunk=(dm.k_star // 4 // 256 + 1) * 256, modulus=89) == RANGE
+    # the whole-procedure entry point applies the same range rule before its first launch
+    rc = L.awe_gemm_exact(fake, ptr, b.I4_IN_I8, ptr, b.I8, 256, 256, 2 ** 20, b.ENC_INT4xINT8_AWE4, 0, ptr, b.C_I32,
+                          ptr, ctypes.c_size_t(1 << 62), None)
+    assert rc == RANGE

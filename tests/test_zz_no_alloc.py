@@ -1,5 +1,6 @@
 """awe_gemm_exact_static -- the entry point for callers that may not allocate device memory --
-against awe_gemm_exact, through the C ABI, bit for bit, on two calls in a row.
+against awe_gemm_exact and against the CPU oracle, through the C ABI, bit for bit, on two calls in a
+row.
 
 Kept in a file that sorts last so that a run stopping at the first failure has already run every
 other test.  The check is self-contained: it passes alone in a fresh process and after the others."""
@@ -7,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import matmul as mm
 from paper_2609_24519_b200 import binding as b
 from paper_2609_24519_b200 import workloads as wl
 
@@ -39,6 +41,10 @@ def test_static_scratch_entry_matches_awe_gemm_exact_twice_in_a_row():
         b.awe_gemm_exact_static(A, a_dt, B, b.I8, w.M, w.N, w.K, enc, modulus, got, out_dt)
         torch.cuda.synchronize()
         assert torch.equal(got, want), w.name
+        exact = mm.matmul_i64(A_np, B_np)                     # the definition: plain int64 product
+        if modulus:
+            exact = mm.mod_symmetric(exact, modulus)
+        assert np.array_equal(got.cpu().numpy().astype(np.int64), exact), w.name
     # the same problem again: stale planes of the previous (different) problem are in the array
     w, enc, out_dt, tdt, modulus, a_dt = cases[0]
     A_np, B_np = wl.make_inputs(w)
@@ -47,7 +53,43 @@ def test_static_scratch_entry_matches_awe_gemm_exact_twice_in_a_row():
     b.awe_gemm_exact_static(A, a_dt, B, b.I8, w.M, w.N, w.K, enc, modulus, got, out_dt)
     torch.cuda.synchronize()
     assert torch.equal(got, _reference(h, A, B, enc, out_dt, tdt, modulus, a_dt))
+    assert np.array_equal(got.cpu().numpy().astype(np.int64), mm.matmul_i64(A_np, B_np))
     b.awe_destroy(h)
+
+
+def test_static_scratch_entry_does_not_wait_for_other_streams_and_replays_from_a_graph():
+    """The call never blocks on the GPU: with a long kernel queue on another stream it returns at once
+    and its product still completes correctly on its own stream.  A warmed-up call recorded into a
+    graph gives the right product on every replay."""
+    w = wl.small("na4", 256, 384, 1024, seed=44)
+    A_np, B_np = wl.make_inputs(w)
+    A, B = torch.from_numpy(A_np).cuda(), torch.from_numpy(B_np).cuda()
+    want = mm.matmul_i64(A_np, B_np)
+    C = torch.zeros((w.M, w.N), dtype=torch.int32, device="cuda")
+    side, busy = torch.cuda.Stream(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        b.awe_gemm_exact_static(A, b.I8, B, b.I8, w.M, w.N, w.K, b.ENC_INT8_AWE6, 0, C, b.C_I32)   # warm-up
+    side.synchronize()
+    big = torch.empty(1 << 28, dtype=torch.uint8, device="cuda")
+    with torch.cuda.stream(busy):
+        for _ in range(200):
+            big.fill_(1)                                       # tens of milliseconds of queued work
+    C.zero_()
+    with torch.cuda.stream(side):
+        b.awe_gemm_exact_static(A, b.I8, B, b.I8, w.M, w.N, w.K, b.ENC_INT8_AWE6, 0, C, b.C_I32)
+    assert not busy.query()                                    # returned while the other stream still runs
+    side.synchronize()
+    assert np.array_equal(C.cpu().numpy(), want)
+    busy.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        b.awe_gemm_exact_static(A, b.I8, B, b.I8, w.M, w.N, w.K, b.ENC_INT8_AWE6, 0, C, b.C_I32)
+    for rep in range(2):
+        A.copy_(torch.from_numpy(np.roll(A_np, rep, axis=0)).cuda())
+        C.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(C.cpu().numpy(), np.roll(want, rep, axis=0))
 
 
 def test_static_scratch_entry_rejects_problems_beyond_its_array():
