@@ -31,7 +31,9 @@ if ROOT not in sys.path:
 METRIC = "effective exact INT8xINT8 TOPS (2*M*N*K / time), AWE 6-GEMM"
 NOMINAL_FP4_TFLOPS = 9000.0          # published dense FP4 peak of one B200 (paper, Section 6.2)
 NOMINAL_FP4_OVER_BF16 = 4.0          # 9.0 / 2.25 PFLOP/s nominal
-GEMM_DRAM_BYTES_8192 = 1646774784 + 356711424   # ncu capture of awe_gemm_kernel at 8192^3, AWE-6
+GEMM_TRAFFIC_JSON = os.path.join(ROOT, "profiles", "awe_gemm_kernel_8192_awe6_traffic.json")
+GEMM_KERNEL_SOURCES = ["awe_gemm.cu", "gemm_common.cuh", "ptx.cuh"]
+BURST_REGION_S = 0.5                 # the power regulator needs about this long to pull the clock down
 MAC_PER_CLK_PER_SM = 16384           # dense FP4: 4 x the 4096 bf16 MAC/clk/SM of the tcgen05 pipe
 
 
@@ -44,15 +46,40 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def gemm_sources_hash():
+    """sha256 over the sources of the product kernel: ties a stored ncu figure to the code it measured."""
+    import hashlib
+    hsh = hashlib.sha256()
+    for f in GEMM_KERNEL_SOURCES:
+        hsh.update(open(os.path.join(ROOT, "paper_2609_24519_b200", "csrc", f), "rb").read())
+    return hsh.hexdigest()[:16]
+
+
+def gemm_dram_traffic(M, N, K, encoding):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one product launch from the committed ncu
+    capture, or None when the capture is of another workload or of older kernel sources."""
+    try:
+        d = json.load(open(GEMM_TRAFFIC_JSON))
+    except Exception:
+        return None, "no capture on file"
+    if (d.get("M"), d.get("N"), d.get("K"), d.get("encoding")) != (M, N, K, encoding):
+        return None, "the capture on file is of another workload"
+    if d.get("sources_sha256_16") != gemm_sources_hash():
+        return None, "kernel sources changed since the capture on file (%s)" % d.get("summary")
+    return int(d["dram_bytes_read"]) + int(d["dram_bytes_write"]), \
+        "dram__bytes_read.sum + dram__bytes_write.sum of one launch at this workload (%s)" % d.get("summary")
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU through NVML while the timed regions run."""
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
                0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting"}
 
     def __init__(self, index: int, uuid: str = ""):
-        self.samples, self.reasons, self.max_mhz, self.power = [], set(), None, []
+        self.by_region, self.max_mhz = {}, None
         self._stop = threading.Event()
         self._active = threading.Event()
+        self._region = None
         self._thread = None
         try:
             import pynvml
@@ -70,32 +97,41 @@ class ClockSampler:
         nv = self._nv
         while not self._stop.is_set():
             if self._active.is_set():
+                rec = self.by_region.setdefault(self._region, {"mhz": [], "reasons": set(), "power": []})
                 try:
-                    self.samples.append(nv.nvmlDeviceGetClockInfo(self._dev, nv.NVML_CLOCK_SM))
+                    rec["mhz"].append(nv.nvmlDeviceGetClockInfo(self._dev, nv.NVML_CLOCK_SM))
                     mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._dev)
                     for bit, name in self.REASONS.items():
                         if mask & bit:
-                            self.reasons.add(name)
-                    self.power.append(nv.nvmlDeviceGetPowerUsage(self._dev) / 1000.0)
+                            rec["reasons"].add(name)
+                    rec["power"].append(nv.nvmlDeviceGetPowerUsage(self._dev) / 1000.0)
                 except Exception:
                     pass
-            time.sleep(0.005)
+            time.sleep(0.001)
 
     def start(self):
         if self._nv is not None:
             self._thread = threading.Thread(target=self._run, daemon=True)
             self._thread.start()
 
-    def region(self, on: bool):
-        (self._active.set if on else self._active.clear)()
+    def region(self, name):
+        """Samples taken from now on belong to region `name`; None pauses sampling."""
+        if name is None:
+            self._active.clear()
+        else:
+            self._region = name
+            self._active.set()
+
+    def summary(self, name):
+        rec = self.by_region.get(name, {"mhz": [], "reasons": set(), "power": []})
+        return {"sm_mhz": statistics.median(rec["mhz"]) if rec["mhz"] else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(rec["reasons"]), "samples": len(rec["mhz"]),
+                "power_w_max": max(rec["power"]) if rec["power"] else None}
 
     def stop(self):
         self._stop.set()
         if self._thread:
             self._thread.join()
-        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples),
-                "power_w_max": max(self.power) if self.power else None}
 
 
 def cpu_oracle_sample(A, B, budget_s: float):
@@ -232,19 +268,21 @@ def main():
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = b.awe_launch_count(h)
     barrier()
-    sampler.region(True)
+    sampler.region("device_resident")
     t_start.record()
     for i in range(args.steps):
         step(evs[i])
     t_end.record()
     barrier()
-    sampler.region(False)
+    sampler.region(None)
     launches = b.awe_launch_count(h) - launches0
     ops = 2.0 * M * N * K
     ms_total, ops_all_ranks = replicas.aggregate(t_start.elapsed_time(t_end), ops * args.steps, dev)
     ms_step = ms_total / args.steps
-    ms_encode = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
-    ms_gemm = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    enc_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    gemm_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    step_ms = [e[0].elapsed_time(e[2]) for e in evs]
+    ms_encode, ms_gemm = statistics.mean(enc_ms), statistics.mean(gemm_ms)
     assert b.awe_last_device_status(h) == (0, 0)
     gemm_mhz = b.awe_last_gemm_clock_mhz(h)       # SM clock measured inside the last timed GEMM launch
 
@@ -258,30 +296,40 @@ def main():
         b.awe_gemm_exact_host(h, Ah, b.I8, Bh, b.I8, M, N, K, enc, 0, Ch, b.C_I32, scratch)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    sampler.region(True)
+    sampler.region("e2e")
     e0.record()
     for _ in range(e2e_steps):
         b.awe_gemm_exact_host(h, Ah, b.I8, Bh, b.I8, M, N, K, enc, 0, Ch, b.C_I32, scratch)
     e1.record()
     barrier()
-    sampler.region(False)
+    sampler.region(None)
     ms_e2e_total, ops_e2e_all = replicas.aggregate(e0.elapsed_time(e1), ops * e2e_steps, dev)
     ms_e2e = ms_e2e_total / e2e_steps
     parity_ok = parity_ok and bool(torch.equal(Ch, C.cpu()))
-    clocks = sampler.stop()
+    sampler.stop()
+    clocks = sampler.summary("device_resident")
     clocks["sm_mhz_in_gemm_kernel"] = gemm_mhz
-    clocks["note"] = ("sm_mhz: NVML samples during the timed regions; sm_mhz_in_gemm_kernel: SM cycles / "
-                      "wall time measured inside the last timed GEMM launch")
+    clocks["e2e_region"] = sampler.summary("e2e")
+    clocks["note"] = ("sm_mhz, reasons, power: NVML samples (1 ms apart) during the device-resident timed region; "
+                      "e2e_region: the same for the host-buffer region; sm_mhz_in_gemm_kernel: SM cycles / wall "
+                      "time measured inside the last timed GEMM launch")
 
     sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
     peaks = measured_peaks()
-    fp4_peak = peaks["bf16_tflops_sustained"] * NOMINAL_FP4_OVER_BF16
+    # Denominator: the peaks file has no FP4 entry, so the measured bf16 figure is scaled by the nominal
+    # fp4 : bf16 ratio -- the burst figure when the timed region is too short for the power regulator to
+    # act, the sustained one for a long region.  Both fractions are printed by name as well.
+    region_s = ms_total * 1e-3
+    burst = region_s < BURST_REGION_S
+    peak_key = "bf16_tflops" if burst else "bf16_tflops_sustained"
+    fp4_peak = peaks[peak_key] * NOMINAL_FP4_OVER_BF16
     gemm_tflops = desc.r * ops / (ms_gemm * 1e-3) / 1e12
     plane_bytes = b.awe_planes_bytes(enc, 0, b.SIDE_A, M, K) + b.awe_planes_bytes(enc, 0, b.SIDE_B, N, K)
     # an FP8 product runs at half the FP4 peak: the peak of a record is its flops over its ideal time
     fp4_equiv = sum(2 if desc.fp8[k] else 1 for k in range(desc.r))
     fmt_scale = desc.r / fp4_equiv  # 1 for FP4-only records
     fp4_peak = fp4_peak * fmt_scale
+    traffic, traffic_note = gemm_dram_traffic(M, N, K, args.encoding)
     line = {
         "metric": METRIC, "value": ops_all_ranks / (ms_total * 1e-3) / 1e12, "unit": "TOPS", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -298,14 +346,17 @@ def main():
                 "steps": e2e_steps, "h2d_bytes_per_step": int(A.nbytes + B.nbytes), "d2h_bytes_per_step": int(M * N * 4)},
         "gpu_launches": int(launches),
         "parity": "3-call path == awe_gemm_exact == host path" if parity_ok else "MISMATCH between entry points",
-        "kernels_ms": {"encode_a_plus_b": ms_encode, "gemm_and_reconstruction": ms_gemm},
+        "kernels_ms": {"encode_a_plus_b": ms_encode, "gemm_and_reconstruction": ms_gemm,
+                       "per_step_stats": {name: {"mean": statistics.mean(v), "median": statistics.median(v), "best": min(v)}
+                                          for name, v in (("encode_a_plus_b", enc_ms), ("gemm_and_reconstruction", gemm_ms),
+                                                          ("step", step_ms))}},
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
-                     "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_BYTES_8192 if (M, N, K, args.encoding) == (8192, 8192, 8192, "awe6") else None,
-                     "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one launch at this workload "
-                                     "(ncu capture with one-pass metrics; summary kept under profiles/)",
+                     "frac": gemm_tflops / fp4_peak, "traffic": traffic, "traffic_note": traffic_note,
                      "kernel": "awe_gemm_kernel", "flops_per_launch": desc.r * ops,
-                     "peak_source": "%s bf16 sustained %.1f TFLOP/s x nominal fp4:bf16 ratio 4" %
-                                    (peaks["source"], peaks["bf16_tflops_sustained"]),
+                     "peak_source": "%s %s %.1f TFLOP/s x nominal fp4:bf16 ratio 4 (timed region %.3f s: %s)" %
+                                    (peaks["source"], peak_key, peaks[peak_key], region_s,
+                                     "burst" if burst else "sustained"),
+                     "frac_of_sustained_peak": gemm_tflops / (peaks["bf16_tflops_sustained"] * NOMINAL_FP4_OVER_BF16 * fmt_scale),
                      "frac_of_nominal_9pflops": gemm_tflops / (NOMINAL_FP4_TFLOPS * fmt_scale),
                      "frac_of_pipe_peak_at_delivered_clock":
                          gemm_tflops / (fmt_scale * MAC_PER_CLK_PER_SM * 2 * sm_count * gemm_mhz * 1e6 / 1e12) if gemm_mhz else None,
@@ -349,6 +400,7 @@ def main():
         torch.cuda.synchronize()
         ctx["base13_9gemm_TOPS"] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
         ctx["base13_equals_awe6"] = bool(torch.equal(C9, C))
+        parity_ok = parity_ok and ctx["base13_equals_awe6"]
         del ws9, C9
         # mixed 2 x FP8 + 1 x FP4 construction (Appendix A) on the same inputs: whole call and its product kernel
         encm = b.ENC_INT8_MIXED_FP8_3
@@ -373,6 +425,7 @@ def main():
         ctx["mixed_2fp8_1fp4_products_ms"] = e0.elapsed_time(e1) / 10
         ctx["mixed_sm_mhz"] = b.awe_last_gemm_clock_mhz(h)
         ctx["mixed_equals_awe6"] = bool(torch.equal(Cm, C))
+        parity_ok = parity_ok and ctx["mixed_equals_awe6"]
         del wsm, Cm, pam, pbm
         # INT8 tensor-core GEMM of the same product (library reference point)
         try:
@@ -386,6 +439,7 @@ def main():
             torch.cuda.synchronize()
             ctx["int8_tensor_core_gemm_TOPS"] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
             ctx["int8_gemm_equals_awe6"] = bool(torch.equal(Ci, C))
+            parity_ok = parity_ok and ctx["int8_gemm_equals_awe6"]
             del Ci
         except Exception as ex:  # library reference point only
             ctx["int8_tensor_core_gemm_TOPS"] = None
@@ -541,6 +595,17 @@ def main():
         same = bool(np.array_equal(c_rows, C[:n_rows].cpu().numpy().astype(np.int64)))
         line["parity"] += ("; GPU rows 0..%d bit-exact vs the CPU oracle" % (n_rows - 1)) if same else \
             "; MISMATCH vs the CPU oracle"
+        parity_ok = parity_ok and same
+        # the textbook (i, j, k) loop nest on one thread, once, at 1024^3
+        from oracle import matmul as om
+        n1 = min(1024, M, N, K)
+        t0 = time.perf_counter()
+        c_naive = om.matmul_i64_ijk(A[:n1, :n1], B[:n1, :n1])
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"]["naive"] = {"value": 2.0 * n1 ** 3 / dt / 1e12, "unit": "TOPS", "cores": 1,
+                                         "kind": "oracle, textbook i-j-k loop nest",
+                                         "sample": "%d^3 corner of the workload (%.1f s)" % (n1, dt)}
+        del c_naive
 
     elif rank == 0:
         line["cpu_baseline"] = None
@@ -549,6 +614,8 @@ def main():
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+    if not parity_ok:
+        raise SystemExit("bench.py: parity mismatch (see the `parity` field)")
 
 
 if __name__ == "__main__":

@@ -312,7 +312,10 @@ awe_status_t awe_fp8_product_raw(awe_handle_t h, const void* planeX_dev, const v
  * matrix at P_dev + k * plane_stride with leading dimension ldp (floats, doubled-integer
  * convention).  Writes C = (sum_k l_k P_k) >> log2 D, or that sum mod m in the symmetric range, to
  * C_dev (leading dimension ldc, type out_dt).  The unfused counterpart of the epilogue of
- * awe_gemm_planes; every P_k must come from a single exact accumulation segment (K <= K*). */
+ * awe_gemm_planes; every P_k must come from a single exact accumulation segment (K <= K*), and
+ * AWE_C_I32 is subject to the same bound as there (D max|a| max|b| K < 2^31; not checked here, since
+ * K is not an argument).  16-byte aligned P_dev and C rows with ldp, ldc, plane_stride multiples of 4
+ * take the vector path. */
 awe_status_t awe_reconstruct(awe_handle_t h, int enc, int modulus, const float* P_dev, int64_t plane_stride,
                              int64_t ldp, int64_t M, int64_t N, void* C_dev, awe_out_dtype_t out_dt, int64_t ldc,
                              void* stream);

@@ -33,6 +33,7 @@ def _load():
         _lib = ctypes.CDLL(build())
         i64, p = ctypes.c_int64, ctypes.c_void_p
         _lib.oracle_matmul_i64.argtypes = [p, p, p, i64, i64, i64]
+        _lib.oracle_matmul_i64_ijk.argtypes = [p, p, p, i64, i64, i64]
         _lib.oracle_matmul_i64_rows.argtypes = [p, p, p, i64, i64, i64, i64]
         _lib.oracle_mod_symmetric.argtypes = [p, i64, i64]
         _lib.oracle_matmul_i64_s16_rows.argtypes = [p, p, p, i64, i64, i64, i64]
@@ -58,6 +59,17 @@ def matmul_i64(A: np.ndarray, B: np.ndarray) -> np.ndarray:
     assert K == K2
     C = np.empty((M, N), dtype=np.int64)
     _load().oracle_matmul_i64(A.ctypes.data, B.ctypes.data, C.ctypes.data, M, N, K)
+    return C
+
+
+def matmul_i64_ijk(A: np.ndarray, B: np.ndarray) -> np.ndarray:
+    """The same product by the textbook (i, j, k) loop nest on one thread."""
+    A, B = _i8(A), _i8(B)
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2
+    C = np.empty((M, N), dtype=np.int64)
+    _load().oracle_matmul_i64_ijk(A.ctypes.data, B.ctypes.data, C.ctypes.data, M, N, K)
     return C
 
 

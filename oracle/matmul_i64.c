@@ -36,6 +36,19 @@ void oracle_matmul_i64(const int8_t* A, const int8_t* B, int64_t* C, int64_t M, 
     }
 }
 
+/* The same definition in its textbook order (i, j, k innermost), on one thread: every entry is one
+ * dot product of a row of A with a column of B.  Timed by the benchmark at 1024^3 as the naive
+ * CPU reference point; also a second, independently ordered check of the loop nest above. */
+void oracle_matmul_i64_ijk(const int8_t* A, const int8_t* B, int64_t* C, int64_t M, int64_t N, int64_t K)
+{
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            int64_t acc = 0;
+            for (int64_t k = 0; k < K; ++k) acc += (int64_t)A[i * K + k] * (int64_t)B[k * N + j];
+            C[i * N + j] = acc;
+        }
+}
+
 /* Rows i0 <= i < i1 only (for sampled checks at sizes where the whole product is too slow). */
 void oracle_matmul_i64_rows(const int8_t* A, const int8_t* B, int64_t* C_rows, int64_t i0, int64_t i1,
                             int64_t N, int64_t K)

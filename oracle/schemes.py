@@ -294,14 +294,52 @@ _K3_PLANES = ((1, 0), (0, 1), (1, -1))
 _D4_ALPHA = ((1, 0), (1, 0), (0, 1), (0, 1))
 _D4_BETA = ((1, 0), (0, 1), (1, 0), (0, 1))
 _mod_cache: Dict[int, Optional[Scheme]] = {}
+K3_MAX_COMPONENT = 4
+
+
+def _k3_general(m: int) -> Optional[Scheme]:
+    """Three products on two limbs with a general third plane p a0 + q a1 (same planes and weights
+    (1, w1) on both sides).  From
+        (a0 + w1 a1)(b0 + w1 b1) = a0 b0 + w1 (a0 b1 + a1 b0) + w1^2 a1 b1,
+        (p a0 + q a1)(p b0 + q b1) = p^2 a0 b0 + p q (a0 b1 + a1 b0) + q^2 a1 b1
+    the coefficients are l3 with l3 p q = w1, l1 = 1 - l3 p^2, l2 = w1^2 - l3 q^2 (all mod m).
+    Candidates in the order (largest plane value, |p| + |q|, p, q, w1); the smallest l3 that solves
+    the congruence is taken."""
+    best = None
+    for p in range(1, K3_MAX_COMPONENT + 1):          # (p, q) and (-p, -q) are the same plane up to sign
+        for q in range(-K3_MAX_COMPONENT, K3_MAX_COMPONENT + 1):
+            if q == 0:
+                continue
+            planes = ((1, 0), (0, 1), (p, q))
+            pairs = [(a0, a1) for a0 in S for a1 in S if p * a0 + q * a1 in S_SET]
+            if len(pairs) < m:
+                continue                               # too few admissible tuples to reach every residue
+            for w1 in range(1, m):
+                if len({(a0 + w1 * a1) % m for a0, a1 in pairs}) < m:
+                    continue
+                l3 = next((l for l in range(m) if (l * p * q - w1) % m == 0), None)
+                if l3 is None:
+                    continue
+                c = _covers(m, (1, w1), planes)
+                assert c is not None
+                key = (c, abs(p) + abs(q), p, q, w1)
+                if best is None or key < best[0]:
+                    best = (key, planes, w1, l3)
+    if best is None:
+        return None
+    (_, _, p, q, _), planes, w1, l3 = best
+    ell = ((1 - l3 * p * p) % m, (w1 * w1 - l3 * q * q) % m, l3 % m)
+    return Scheme(f"mod{m}_3g", (1, w1), (1, w1), planes, planes, ell, modulus=m)
 
 
 def mod_scheme(m: int) -> Optional[Scheme]:
-    """Residue scheme for modulus m (Section 5.3), cheapest of three constructions:
+    """Residue scheme for modulus m (Section 5.3), cheapest of these constructions:
 
       1 product : one limb a = x (mod m), only for the moduli S covers by itself;
       3 products: limbs (a0, a1), planes (a0, a1, a0 - a1) on both sides, from
                   xy = (1 + w1) a0 b0 + (w1^2 + w1) a1 b1 - w1 (a0 - a1)(b0 - b1);
+                  where no weight works with that third plane, any third plane p a0 + q a1 with
+                  |p|, |q| <= 4 (_k3_general);
       4 products: limbs (a0, a1), all four limb pairs, coefficients (1, w1, w1, w1^2).
     The paper prints no residue table; these are constructions of Definition 4.1 relaxed
     to a congruence, each checked exhaustively by the tests."""
@@ -315,6 +353,9 @@ def mod_scheme(m: int) -> Optional[Scheme]:
         if w1 is not None:
             ell = ((1 + w1) % m, (w1 * w1 + w1) % m, (-w1) % m)
             sch = Scheme(f"mod{m}_3", (1, w1), (1, w1), _K3_PLANES, _K3_PLANES, ell, modulus=m)
+    if sch is None and 2 <= m <= 4 * 133:
+        # at most 133 limb pairs are admissible with a third plane, so larger moduli cannot be covered
+        sch = _k3_general(m)
     if sch is None and m >= 2:
         w1 = _best_w1(m, ((1, 0), (0, 1)))
         if w1 is not None:

@@ -95,7 +95,7 @@ struct awe_ctx {
     // copy engines of the host-buffer entry point: one stream per direction and the events that
     // order them against the caller's stream (created on first use)
     static constexpr int kMaxHostChunks = 16;   // row chunks of A and C
-    static constexpr int kMaxHostColBlocks = 4;  // column blocks of B and C
+    static constexpr int kMaxHostColBlocks = 8;  // column blocks of B and C
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_done = nullptr;
     cudaEvent_t ev_a[kMaxHostChunks] = {nullptr}, ev_bcol[kMaxHostColBlocks] = {nullptr};

@@ -346,6 +346,63 @@ bool make_mod(int m, Scheme* out) {
         *out = s;
         return true;
     }
+    // three products with a general third plane p a0 + q a1 (|p|, |q| <= 4, p > 0: the sign of a plane
+    // is arbitrary), for the moduli no weight covers with a0 - a1.  From
+    //   (a0 + w1 a1)(b0 + w1 b1) = a0 b0 + w1 (a0 b1 + a1 b0) + w1^2 a1 b1
+    //   (p a0 + q a1)(p b0 + q b1) = p^2 a0 b0 + p q (a0 b1 + a1 b0) + q^2 a1 b1
+    // the coefficients are l3 with l3 p q = w1, l1 = 1 - l3 p^2, l2 = w1^2 - l3 q^2 (mod m).  Candidates
+    // are ranked by (largest plane value, |p| + |q|, p, q, w1).
+    {
+        bool in_s[64] = {false};
+        for (int x : kS) in_s[x + 32] = true;
+        int bp = 0, bq = 0, bw = 0, bl3 = 0, bc = 1 << 30, bsum = 0;
+        for (int pp = 1; pp <= 4; ++pp)
+            for (int qq = -4; qq <= 4; ++qq) {
+                if (qq == 0) continue;
+                int admissible = 0;
+                for (int a0 : kS)
+                    for (int a1 : kS) {
+                        const int t = pp * a0 + qq * a1;
+                        if (t >= -12 && t <= 12 && in_s[t + 32]) ++admissible;
+                    }
+                if (admissible < m) continue;  // too few admissible limb pairs to reach every residue
+                const int pl[3][kMaxLimbs] = {{1, 0}, {0, 1}, {pp, qq}};
+                for (int w1 = 1; w1 < m; ++w1) {
+                    int l3 = -1;
+                    for (int l = 0; l < m && l3 < 0; ++l)
+                        if ((((l * pp * qq - w1) % m) + m) % m == 0) l3 = l;
+                    if (l3 < 0) continue;
+                    const int c = two_limb_cover(m, w1, 3, pl);
+                    if (c < 0) continue;
+                    const int sum = pp + std::abs(qq);
+                    // lexicographic comparison of (c, |p|+|q|, p, q, w1) with the best so far
+                    const int cand[5] = {c, sum, pp, qq, w1}, cur[5] = {bc, bsum, bp, bq, bw};
+                    bool better = bw == 0;
+                    for (int i = 0; i < 5 && !better; ++i) {
+                        if (cand[i] < cur[i]) better = true;
+                        else if (cand[i] > cur[i]) break;
+                    }
+                    if (better) {
+                        bc = c; bsum = sum; bp = pp; bq = qq; bw = w1; bl3 = l3;
+                    }
+                }
+            }
+        if (bw) {
+            s.p = s.q = 2;
+            s.r = 3;
+            s.w[0] = s.v[0] = 1;
+            s.w[1] = s.v[1] = bw;
+            const int pl[3][kMaxLimbs] = {{1, 0}, {0, 1}, {bp, bq}};
+            for (int k = 0; k < 3; ++k)
+                for (int i = 0; i < 2; ++i) s.alpha[k][i] = s.beta[k][i] = pl[k][i];
+            auto modm = [m](long long x) { return (int)(((x % m) + m) % m); };
+            s.ell[0] = modm(1 - (long long)bl3 * bp * bp);
+            s.ell[1] = modm((long long)bw * bw - (long long)bl3 * bq * bq);
+            s.ell[2] = modm(bl3);
+            *out = s;
+            return true;
+        }
+    }
     // four products on two limbs: all limb pairs, coefficients (1, w1, w1, w1^2)
     const int d2[2][kMaxLimbs] = {{1, 0}, {0, 1}};
     for (int w1 = 1; w1 < m; ++w1) {

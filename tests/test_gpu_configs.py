@@ -1,6 +1,7 @@
 """The benchmark configurations at full size, through the same three C-ABI calls bench.py times.
-The CPU oracle checks sampled rows (it computes them one by one); whole-matrix checks use
-properties that hold at any size: every INT8 encoding must give the same matrix, and the
+Configuration 2 and the headline shape are compared with the CPU oracle over the WHOLE matrix (the
+plain int64 product takes seconds there); the larger ones on sampled rows the oracle computes one by
+one, plus properties that hold at any size: every INT8 encoding must give the same matrix, and the
 residue of the exact product must equal the residue product."""
 import numpy as np
 import pytest
@@ -51,7 +52,7 @@ def test_config2_awe6_and_base13_on_identical_inputs():
     w = wl.config2()
     A, B = wl.make_inputs(w)
     C6 = run_three_calls(w, A, B, b.ENC_INT8_AWE6, b.C_I32)
-    assert sampled_rows_match(C6, A, B, 24, 2)
+    assert np.array_equal(C6.cpu().numpy(), mm.matmul_i64(A, B))          # every entry, against the definition
     C9 = run_three_calls(w, A, B, b.ENC_INT8_BASE13_9, b.C_I32)
     assert torch.equal(C6, C9)
     Calt = run_three_calls(w, A, B, b.ENC_INT8_AWE6_ALT, b.C_I32)
@@ -95,5 +96,8 @@ def test_headline_8192_int8():
     w = wl.headline()
     A, B = wl.make_inputs(w)
     C = run_three_calls(w, A, B, b.ENC_INT8_AWE6, b.C_I32)
-    assert sampled_rows_match(C, A, B, 16, 6)
+    # every entry against the definition, in row bands so the int64 reference stays small
+    got = C.cpu().numpy()
+    for r0 in range(0, w.M, 1024):
+        assert np.array_equal(got[r0:r0 + 1024], mm.matmul_i64_rows(A, B, r0, min(w.M, r0 + 1024))), r0
     assert torch.equal(C, run_three_calls(w, A, B, b.ENC_INT8_BASE13_9, b.C_I32))

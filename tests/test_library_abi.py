@@ -83,7 +83,7 @@ def test_tables_match_the_oracle_tables(b):
     assert not lut[2:255].any()                                   # non-ternary bytes are read as 0
     assert np.array_equal(b.awe_encoding_lut(b.ENC_TERNARY_INT8_3, 0, b.SIDE_B)[idx],
                           pl.plane_lut(sc.TERNARY3, "B", -128, 127))
-    for m in rns.RNS_SET_FP64 + (2, 10, 37, 91, 100, 169):
+    for m in rns.RNS_SET_FP64 + (2, 10, 37, 60, 66, 72, 91, 100, 169):
         s = sc.mod_scheme(m)
         d = b.awe_encoding_info(b.ENC_MOD_M, m)
         assert d.r == s.r and list(d.ell)[:d.r] == list(s.ell) and d.modulus == m

@@ -23,10 +23,12 @@ def test_c_loop_nest_against_python_integers_and_numpy():
         C = mm.matmul_i64(A, B)
         assert np.array_equal(C, _py_matmul(A, B))
         assert np.array_equal(C, mm.matmul_i64_numpy(A, B))
+        assert np.array_equal(mm.matmul_i64_ijk(A, B), _py_matmul(A, B))
     A = rng.integers(-128, 128, (70, 300), dtype=np.int8)
     B = rng.integers(-128, 128, (300, 50), dtype=np.int8)
     assert np.array_equal(mm.matmul_i64(A, B), mm.matmul_i64_numpy(A, B))
     assert np.array_equal(mm.matmul_i64_rows(A, B, 13, 29), mm.matmul_i64_numpy(A, B)[13:29])
+    assert np.array_equal(mm.matmul_i64_ijk(A, B), mm.matmul_i64_numpy(A, B))
 
 
 def test_closed_forms():
@@ -43,6 +45,7 @@ def test_closed_forms():
     A = np.array([[1, 2], [3, 4]], dtype=np.int8)
     Bm = np.array([[0, 1], [1, 1]], dtype=np.int8)
     assert mm.matmul_i64(A, Bm).tolist() == [[2, 3], [4, 7]]
+    assert mm.matmul_i64_ijk(A, Bm).tolist() == [[2, 3], [4, 7]]
 
 
 def test_int16_product_against_numpy_and_python():

@@ -47,7 +47,7 @@ def test_symmetric_range():
             assert lo <= y <= hi and (x - y) % m == 0
 
 
-@pytest.mark.parametrize("m", rns.RNS_SET_FP64)
+@pytest.mark.parametrize("m", rns.RNS_SET_FP64 + (10, 37, 60, 62, 66, 72, 91, 100, 169))
 def test_all_residue_pairs(m):
     """Every residue pair: planes in S, limbs in S, value congruent, and
     sum_k l_k P_k == x y (mod m) with integer coefficients."""
@@ -79,6 +79,29 @@ def test_three_product_expansion_by_hand():
         assert (full - got) % 41 == 0
 
 
+def test_three_product_moduli_of_the_two_limb_family():
+    """Which moduli cost three products when both sides use limbs (a0, a1) and planes a0, a1 and one
+    third plane p a0 + q a1 with |p|, |q| <= 4: 10, 12, every modulus from 14 to 67, and
+    69, 71, 72, 73, 75, ..., 91 (odd) -- 69 moduli, none above 91.  The third plane a0 - a1 serves all of
+    them except 60, 62, 66 and 72, which need 2 a0 - a1.  (Section 5.3 speaks of 82 such moduli without
+    printing them: parity with that list is unpinned.)"""
+    three = [m for m in range(2, 170) if sc.mod_scheme(m) is not None and sc.mod_scheme(m).r == 3]
+    assert three == [10, 12] + list(range(14, 68)) + [69, 71, 72, 73] + list(range(75, 92, 2))
+    assert len(three) == 69
+    general = [m for m in three if sc.mod_scheme(m).alpha[2] != (1, -1)]
+    assert general == [60, 62, 66, 72]
+    for m in general:
+        s = sc.mod_scheme(m)
+        assert s.alpha == s.beta == ((1, 0), (0, 1), (2, -1)) and sc.coefficient_identity_holds(s)
+    # the identity behind the coefficients, written out by hand for m = 60:
+    # (a0 + w a1)(b0 + w b1) = l1 a0 b0 + l2 a1 b1 + l3 (2 a0 - a1)(2 b0 - b1)  (mod 60)
+    s = sc.mod_scheme(60)
+    w = s.w[1]
+    for a0, a1, b0, b1 in [(1, 2, 3, 4), (-6, 3, 8, -2), (12, 8, -12, -8)]:
+        got = s.ell[0] * a0 * b0 + s.ell[1] * a1 * b1 + s.ell[2] * (2 * a0 - a1) * (2 * b0 - b1)
+        assert ((a0 + w * a1) * (b0 + w * b1) - got) % 60 == 0
+
+
 def test_rns_set_for_the_fp64_significand():
     g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "paper_constants.json")))["rns_fp64"]
     sel = list(rns.RNS_SET_FP64)
@@ -101,7 +124,7 @@ def test_integer_program_reaches_the_same_total():
 
 def test_one_more_three_product_modulus_would_give_the_printed_total():
     """Sensitivity of the unpinned total: the program returns the paper's 59 as soon as 95 or 97 costs
-    three products, and no two-limb scheme with a third plane p a0 + q a1 (|p|, |q| <= 2) reaches them."""
+    three products, and no two-limb scheme with a third plane p a0 + q a1 (|p|, |q| <= 4) reaches them."""
     g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "paper_constants.json")))["rns_fp64"]
     costs = rns.cost_table(170)
     assert costs[95] == costs[97] == 4
@@ -110,7 +133,7 @@ def test_one_more_three_product_modulus_would_give_the_printed_total():
         for m in extra:
             c2[m] = 3
         assert rns.select_moduli(c2)[0] == g["awe_products"]
-    for p, q in ((1, -1), (1, 1), (1, 2), (1, -2), (2, 1), (2, -1)):
+    for p, q in [(p, q) for p in range(1, 5) for q in range(-4, 5) if q]:
         T = [(a0, a1) for a0 in sc.S for a1 in sc.S if (p * a0 + q * a1) in sc.S_SET]
         assert len(T) <= 133
         for m in (95, 97):
