@@ -204,11 +204,12 @@ awe_status_t awe_gemm_exact(awe_handle_t h, const void* A_dev, awe_in_dtype_t a_
 /* Same product with HOST operands and result: copies A_host and B_host to the device, runs
  * awe_gemm_exact, copies C back to C_host and waits for the stream, so C_host is valid on return.
  * scratch_dev must hold awe_workspace_bytes + awe_host_staging_bytes bytes (256-B aligned).
- * For M >= 2048 the product is processed in blocks (rows of A and C in up to 16 chunks and, from
- * M, N >= 4096, columns of B and C in up to 4 blocks) so that the copies to the device, the kernels
- * and the copies back overlap; the copies run on two streams owned by the handle (created on the
- * first call) that are ordered after and before `stream` with events.  Pinned host memory is needed
- * for that overlap; pageable memory works but serialises. */
+ * For M >= 2048 the product is processed in blocks (row chunks of A; from N >= 4096 also column blocks
+ * of B, uploaded alternately so that about as many rows of A as columns of B are on the device, each
+ * arrival followed by one launch for the rectangle of C it completes and one copy back) so that the
+ * copies to the device, the kernels and the copies back overlap; the copies run on two streams owned by
+ * the handle (created on the first call) that are ordered after and before `stream` with events.
+ * Pinned host memory is needed for that overlap; pageable memory works but serialises. */
 awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, awe_in_dtype_t a_dt, const void* B_host,
                                  awe_in_dtype_t b_dt, int64_t M, int64_t N, int64_t K, int enc, int modulus,
                                  void* C_host, awe_out_dtype_t out_dt, void* scratch_dev, size_t scratch_bytes,

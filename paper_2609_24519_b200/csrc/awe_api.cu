@@ -106,11 +106,6 @@ awe_status_t device_lut(awe_ctx* h, int enc, int modulus, awe_side_t side, awe_i
 }
 }  // namespace awe
 
-// rows of all stored planes of a side, in units of the E2M1 pitch (an E4M3 plane counts twice)
-static int t_planes(const awe_encoding_desc& d, awe_side_t side) {
-    return side == AWE_SIDE_A ? plane_units(d.plane_bits_a, d.n_planes_a) : plane_units(d.plane_bits_b, d.n_planes_b);
-}
-
 static size_t out_elem_bytes(awe_out_dtype_t t) { return t == AWE_C_I64 ? 8 : (t == AWE_C_RES_I16 ? 2 : 4); }
 
 extern "C" size_t awe_host_staging_bytes(int enc, int modulus, int64_t M, int64_t N, int64_t K,
@@ -194,20 +189,43 @@ extern "C" awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, 
         (s = device_lut(h, enc, modulus, AWE_SIDE_B, b_dt, st, &lut)) != AWE_OK)
         return s;
 
-    // The product is cut into blocks -- rows of A and C into up to 16 chunks, columns of B and C into up
-    // to 4 blocks, about 2048 x 2048 each (one wave of tile pairs per launch) -- so that the copies to the
-    // device, the kernels and the copies back overlap (the two copy directions run on their own
-    // streams).  The result is twice the bytes of the operands, so the copy back is the long pole: it
-    // starts after one column block of B and one row chunk of A have arrived.  Small problems go
-    // through in one piece.
-    int chunks = (int)std::min<int64_t>(awe_ctx::kMaxHostChunks, M / 2048);
-    int col_blocks = (int)std::min<int64_t>(awe_ctx::kMaxHostColBlocks, N / 2048);
-    if (chunks < 2) {  // few rows: row chunks of 1024 still overlap the copies, without column blocks
-        chunks = (int)std::min<int64_t>(awe_ctx::kMaxHostChunks, M / 1024);
-        col_blocks = 1;
+    // The product is cut into blocks so that the copies to the device, the kernels and the copies back
+    // overlap (the two copy directions run on their own streams).  The result is twice the bytes of the
+    // operands, so the copy back is the long pole: it should start early and never wait.  With a rows
+    // of A and b columns of B on the device, a x b entries of C can be computed, so the uploads alternate
+    // between row chunks of A and column blocks of B to keep a and b about equal (column block 0 first,
+    // small row chunks at the start so that the first block of C leaves after about 0.4 ms).  Each
+    // arrival makes one new rectangle of C computable -- the new rows against all columns present, or
+    // all rows present against the new columns: one launch on planes that every chunk is encoded into
+    // in place, and one two-dimensional copy back.  Small problems go through in one piece.
+    int64_t row_edge[awe_ctx::kMaxHostChunks + 1], col_edge[awe_ctx::kMaxHostColBlocks + 1];
+    int n_row = 0, n_col = 0;
+    auto cut = [](int64_t total, const int64_t* first, int n_first, int64_t rest, int max_parts, int64_t* edge) {
+        int n = 0;
+        int64_t at = 0;
+        edge[0] = 0;
+        while (at < total) {
+            int64_t step = n < n_first ? first[n] : rest;
+            // the last part takes what is left (also when the table of parts is used up)
+            if (n + 1 == max_parts || total - at < step + step / 2) step = total - at;
+            at += step;
+            edge[++n] = at;
+        }
+        return n;
+    };
+    if (M >= 2048 && N >= 4096) {
+        const int64_t rows_first[5] = {512, 512, 1024, 1024, 1024}, cols_first[3] = {2048, 1024, 1024};
+        n_row = cut(M, rows_first, 5, 2048, awe_ctx::kMaxHostChunks, row_edge);
+        n_col = cut(N, cols_first, 3, 2048, awe_ctx::kMaxHostColBlocks, col_edge);
+    } else {
+        // few rows or columns: row chunks of at least 1024 still overlap the copies, no column blocks
+        const int chunks = (int)std::max<int64_t>(1, std::min<int64_t>(awe_ctx::kMaxHostChunks, M / 1024));
+        const int64_t per = chunks == 1 ? M : round_up((M + chunks - 1) / chunks, 256);
+        n_row = cut(M, nullptr, 0, per, awe_ctx::kMaxHostChunks, row_edge);
+        n_col = 1;
+        col_edge[0] = 0;
+        col_edge[1] = N;
     }
-    if (chunks < 2) chunks = 1;
-    if (col_blocks < 2) col_blocks = 1;
     if (!h->copy_in) {
         bool ok = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
@@ -220,81 +238,78 @@ extern "C" awe_status_t awe_gemm_exact_host(awe_handle_t h, const void* A_host, 
         if (!ok) return AWE_ERR_CUDA;
     }
 #define AWE_CU(x) do { if ((x) != cudaSuccess) return AWE_ERR_CUDA; } while (0)
-    const int64_t pitch = plane_pitch_bytes(K);
-    const int64_t units_a = t_planes(d, AWE_SIDE_A), units_b = t_planes(d, AWE_SIDE_B);
     uint8_t* pa = base;
     uint8_t* pb = base + round_up((int64_t)awe_planes_bytes(enc, modulus, AWE_SIDE_A, M, K), 256);
-    const int64_t rows_per_chunk = chunks == 1 ? M : round_up((M + chunks - 1) / chunks, 256);
-    const int64_t cols_per_block = col_blocks == 1 ? N : round_up((N + col_blocks - 1) / col_blocks, 256);
-    const int n_row = (int)((M + rows_per_chunk - 1) / rows_per_chunk);
-    const int n_col = (int)((N + cols_per_block - 1) / cols_per_block);
     const int64_t nib_b = in_elem_nibbles(b_dt);  // half-bytes per element of B
     AWE_CU(cudaEventRecord(h->ev_start, st));
     AWE_CU(cudaStreamWaitEvent(h->copy_in, h->ev_start, 0));
     AWE_CU(cudaStreamWaitEvent(h->copy_out, h->ev_start, 0));
-    // Order of the copies to the device: column block 0 of B, the row chunks of A (the copy back of the
-    // first block column keeps pace with them), then the other column blocks of B.
-    auto upload_b = [&](int j) -> awe_status_t {
-        const int64_t c0 = (int64_t)j * cols_per_block, cols = std::min(cols_per_block, N - c0);
-        if (n_col == 1) {
-            AWE_CU(cudaMemcpyAsync(dB, B_host, (size_t)in_bytes(b_dt, K * N), cudaMemcpyHostToDevice, h->copy_in));
-        } else {
-            AWE_CU(cudaMemcpy2DAsync(dB + c0 * nib_b / 2, (size_t)(N * nib_b / 2), (const uint8_t*)B_host + c0 * nib_b / 2,
-                                     (size_t)(N * nib_b / 2), (size_t)(cols * nib_b / 2), (size_t)K,
-                                     cudaMemcpyHostToDevice, h->copy_in));
+    // Order of arrival: column block 0, then whichever operand has fewer rows (columns) on the device.
+    struct Arrival { bool is_a; int index; };
+    Arrival order[awe_ctx::kMaxHostChunks + awe_ctx::kMaxHostColBlocks];
+    int n_order = 0;
+    {
+        int i = 0, j = 0;
+        order[n_order++] = {false, j++};
+        while (i < n_row || j < n_col) {
+            const bool take_a = i < n_row && (j >= n_col || row_edge[i] < col_edge[j]);
+            order[n_order++] = take_a ? Arrival{true, i++} : Arrival{false, j++};
         }
-        AWE_CU(cudaEventRecord(h->ev_bcol[j], h->copy_in));
-        return AWE_OK;
-    };
-    auto upload_a = [&](int i) -> awe_status_t {
-        const int64_t r0 = (int64_t)i * rows_per_chunk, rows = std::min(rows_per_chunk, M - r0);
-        AWE_CU(cudaMemcpyAsync(dA + (size_t)in_bytes(a_dt, r0 * K), (const uint8_t*)A_host + (size_t)in_bytes(a_dt, r0 * K),
-                               (size_t)in_bytes(a_dt, rows * K), cudaMemcpyHostToDevice, h->copy_in));
-        AWE_CU(cudaEventRecord(h->ev_a[i], h->copy_in));
-        return AWE_OK;
-    };
-    if ((s = upload_b(0)) != AWE_OK) return s;
-    for (int i = 0; i < n_row; ++i)
-        if ((s = upload_a(i)) != AWE_OK) return s;
-    for (int j = 1; j < n_col; ++j)
-        if ((s = upload_b(j)) != AWE_OK) return s;
-    for (int j = 0; j < n_col; ++j) {
-        const int64_t c0 = (int64_t)j * cols_per_block, cols = std::min(cols_per_block, N - c0);
-        uint8_t* pb_j = pb + (size_t)units_b * (size_t)c0 * pitch;  // this block's own plane set
-        AWE_CU(cudaStreamWaitEvent(st, h->ev_bcol[j], 0));
-        if ((s = awe_encode(h, enc, modulus, AWE_SIDE_B, dB + c0 * nib_b / 2, b_dt, AWE_ROWMAJOR_KxR, cols, K, N, pb_j,
-                            stream)) != AWE_OK)
-            return s;
-        for (int i = 0; i < n_row; ++i) {
-            const int64_t r0 = (int64_t)i * rows_per_chunk, rows = std::min(rows_per_chunk, M - r0);
-            uint8_t* pa_i = pa + (size_t)units_a * (size_t)r0 * pitch;
-            if (j == 0) {
-                AWE_CU(cudaStreamWaitEvent(st, h->ev_a[i], 0));
-                if ((s = awe_encode(h, enc, modulus, AWE_SIDE_A, dA + (size_t)in_bytes(a_dt, r0 * K), a_dt, AWE_ROWMAJOR_RxK,
-                                    rows, K, K, pa_i, stream)) != AWE_OK)
-                    return s;
-            }
-            uint8_t* c_blk = dC + ((size_t)r0 * N + c0) * elem;
-            if ((s = awe_gemm_planes(h, enc, modulus, pa_i, pb_j, rows, cols, K, c_blk, out_dt, N, 0, stream)) != AWE_OK)
-                return s;
-            // Copy back: block column 0 goes chunk by chunk, so the first bytes leave as early as possible
-            // (its products keep pace with the arrival of A); a later block column is complete long before
-            // the copy of the previous one ends, and goes back as one two-dimensional copy (every copy
-            // costs a gap of some 15 us on the copy stream).
-            const bool per_chunk = j <= 1 || n_col == 1;
-            if (!per_chunk && i + 1 < n_row) continue;
-            cudaEvent_t done = h->ev_c[j * awe_ctx::kMaxHostChunks + i];
-            AWE_CU(cudaEventRecord(done, st));
-            AWE_CU(cudaStreamWaitEvent(h->copy_out, done, 0));
-            const int64_t rr0 = per_chunk ? r0 : 0, rrows = per_chunk ? rows : M;
-            uint8_t* c_dev = dC + ((size_t)rr0 * N + c0) * elem;
-            uint8_t* c_host = (uint8_t*)C_host + ((size_t)rr0 * N + c0) * elem;
+    }
+    for (int o = 0; o < n_order; ++o) {
+        if (order[o].is_a) {
+            const int64_t r0 = row_edge[order[o].index], rows = row_edge[order[o].index + 1] - r0;
+            AWE_CU(cudaMemcpyAsync(dA + (size_t)in_bytes(a_dt, r0 * K), (const uint8_t*)A_host + (size_t)in_bytes(a_dt, r0 * K),
+                                   (size_t)in_bytes(a_dt, rows * K), cudaMemcpyHostToDevice, h->copy_in));
+            AWE_CU(cudaEventRecord(h->ev_a[order[o].index], h->copy_in));
+        } else {
+            const int64_t c0 = col_edge[order[o].index], cols = col_edge[order[o].index + 1] - c0;
             if (n_col == 1) {
-                AWE_CU(cudaMemcpyAsync(c_host, c_dev, (size_t)rrows * N * elem, cudaMemcpyDeviceToHost, h->copy_out));
+                AWE_CU(cudaMemcpyAsync(dB, B_host, (size_t)in_bytes(b_dt, K * N), cudaMemcpyHostToDevice, h->copy_in));
             } else {
-                AWE_CU(cudaMemcpy2DAsync(c_host, (size_t)N * elem, c_dev, (size_t)N * elem, (size_t)cols * elem,
-                                         (size_t)rrows, cudaMemcpyDeviceToHost, h->copy_out));
+                AWE_CU(cudaMemcpy2DAsync(dB + c0 * nib_b / 2, (size_t)(N * nib_b / 2), (const uint8_t*)B_host + c0 * nib_b / 2,
+                                         (size_t)(N * nib_b / 2), (size_t)(cols * nib_b / 2), (size_t)K,
+                                         cudaMemcpyHostToDevice, h->copy_in));
             }
+            AWE_CU(cudaEventRecord(h->ev_bcol[order[o].index], h->copy_in));
+        }
+    }
+    // C rows [r0, r0 + rows) x columns [c0, c0 + cols): product on the planes present, then the copy back
+    auto region = [&](int slot, int64_t r0, int64_t rows, int64_t c0, int64_t cols) -> awe_status_t {
+        if (rows <= 0 || cols <= 0) return AWE_OK;
+        uint8_t* c_dev = dC + ((size_t)r0 * N + c0) * elem;
+        awe_status_t rs = gemm_planes_window(h, enc, modulus, PlaneWindow{pa, M, r0}, PlaneWindow{pb, N, c0}, rows, cols, K,
+                                             c_dev, out_dt, N, 0, stream);
+        if (rs != AWE_OK) return rs;
+        AWE_CU(cudaEventRecord(h->ev_c[slot], st));
+        AWE_CU(cudaStreamWaitEvent(h->copy_out, h->ev_c[slot], 0));
+        uint8_t* c_host = (uint8_t*)C_host + ((size_t)r0 * N + c0) * elem;
+        if (cols == N) {
+            AWE_CU(cudaMemcpyAsync(c_host, c_dev, (size_t)rows * N * elem, cudaMemcpyDeviceToHost, h->copy_out));
+        } else {
+            AWE_CU(cudaMemcpy2DAsync(c_host, (size_t)N * elem, c_dev, (size_t)N * elem, (size_t)cols * elem, (size_t)rows,
+                                     cudaMemcpyDeviceToHost, h->copy_out));
+        }
+        return AWE_OK;
+    };
+    int64_t a_done = 0, b_done = 0;
+    for (int o = 0; o < n_order; ++o) {
+        if (order[o].is_a) {
+            const int64_t r0 = row_edge[order[o].index], rows = row_edge[order[o].index + 1] - r0;
+            AWE_CU(cudaStreamWaitEvent(st, h->ev_a[order[o].index], 0));
+            if ((s = encode_window(h, enc, modulus, AWE_SIDE_A, dA + (size_t)in_bytes(a_dt, r0 * K), a_dt, AWE_ROWMAJOR_RxK,
+                                   rows, K, K, PlaneWindow{pa, M, r0}, stream)) != AWE_OK)
+                return s;
+            if ((s = region(o, r0, rows, 0, b_done)) != AWE_OK) return s;
+            a_done = r0 + rows;
+        } else {
+            const int64_t c0 = col_edge[order[o].index], cols = col_edge[order[o].index + 1] - c0;
+            AWE_CU(cudaStreamWaitEvent(st, h->ev_bcol[order[o].index], 0));
+            if ((s = encode_window(h, enc, modulus, AWE_SIDE_B, dB + c0 * nib_b / 2, b_dt, AWE_ROWMAJOR_KxR, cols, K, N,
+                                   PlaneWindow{pb, N, c0}, stream)) != AWE_OK)
+                return s;
+            if ((s = region(o, 0, a_done, c0, cols)) != AWE_OK) return s;
+            b_done = c0 + cols;
         }
     }
     AWE_CU(cudaEventRecord(h->ev_done, h->copy_out));

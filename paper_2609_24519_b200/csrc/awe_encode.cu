@@ -120,10 +120,11 @@ __device__ __forceinline__ void encode32_store(const unsigned char* lut_s, uint3
 // Mixed-format record (2 x FP8 + 1 x FP4, Appendix A): the table word of an input byte carries the
 // E4M3 bytes of planes 0 and 1 in bytes 0 and 1 and the E2M1 code of plane 2 in the low nibble of
 // byte 2.  32 consecutive elements of a row give 32 bytes of each E4M3 plane and 16 of the E2M1
-// plane.  Plane 0 starts at `planes`, plane 1 after R rows of 2*pitch bytes, plane 2 after that.
+// plane.  Row 0 of plane 0 is at `planes`, plane 1 follows 2 * plane_stride bytes later (plane_stride
+// counts E2M1 rows of pitch bytes, an E4M3 row is twice as long), row 0 of plane 2 is at `planes4`.
 __device__ __forceinline__ void encode32_store_mixed(const unsigned char* lut_s, uint32_t slot,
-                                                     const uint32_t (&in)[8], uint8_t* planes, int64_t R, int64_t row,
-                                                     int64_t k0, int64_t pitch) {
+                                                     const uint32_t (&in)[8], uint8_t* planes, uint8_t* planes4,
+                                                     int64_t plane_stride, int64_t row, int64_t k0, int64_t pitch) {
     uint32_t p0[8], p1[8], p2[4];
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
@@ -145,8 +146,8 @@ __device__ __forceinline__ void encode32_store_mixed(const unsigned char* lut_s,
     }
     const int64_t pitch8 = 2 * pitch;
     uint8_t* d0 = planes + row * pitch8 + k0;
-    uint8_t* d1 = d0 + R * pitch8;
-    uint8_t* d2 = planes + 2 * R * pitch8 + row * pitch + k0 / 2;
+    uint8_t* d1 = d0 + 2 * plane_stride;
+    uint8_t* d2 = planes4 + row * pitch + k0 / 2;
     *reinterpret_cast<uint4*>(d0) = make_uint4(p0[0], p0[1], p0[2], p0[3]);
     *reinterpret_cast<uint4*>(d0 + 16) = make_uint4(p0[4], p0[5], p0[6], p0[7]);
     *reinterpret_cast<uint4*>(d1) = make_uint4(p1[0], p1[1], p1[2], p1[3]);
@@ -161,7 +162,8 @@ __device__ __forceinline__ void encode32_store_mixed(const unsigned char* lut_s,
 template <int NP, bool kMixed = false, bool kPacked = false>
 __global__ void __launch_bounds__(kEncThreads)
 encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld, const uint64_t* __restrict__ lut_g,
-                  uint8_t* __restrict__ planes, int64_t pitch, int64_t plane_stride, int vec_ok) {
+                  uint8_t* __restrict__ planes, uint8_t* __restrict__ planes4, int64_t pitch, int64_t plane_stride,
+                  int vec_ok) {
     extern __shared__ __align__(128) unsigned char lut_s[];
     load_lut<NP>(lut_s, lut_g);
     const int lane = threadIdx.x & 31;
@@ -216,7 +218,7 @@ encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
                 in[i] = word;
             }
         }
-        if (kMixed) encode32_store_mixed(lut_s, slot, in, planes, R, row, k0, pitch);
+        if (kMixed) encode32_store_mixed(lut_s, slot, in, planes, planes4, plane_stride, row, k0, pitch);
         else encode32_store<NP>(lut_s, slot, in, planes + row * pitch + k0 / 2, plane_stride);
     }
 }
@@ -231,7 +233,8 @@ encode_rxk_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
 template <int NP, bool kMixed = false, bool kPacked = false>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kxr_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld, const uint64_t* __restrict__ lut_g,
-                  uint8_t* __restrict__ planes, int64_t pitch, int64_t plane_stride, int vec_ok) {
+                  uint8_t* __restrict__ planes, uint8_t* __restrict__ planes4, int64_t pitch, int64_t plane_stride,
+                  int vec_ok) {
     extern __shared__ __align__(128) unsigned char lut_s[];
     load_lut<NP>(lut_s, lut_g);
     const int lane = threadIdx.x & 31;
@@ -297,7 +300,7 @@ encode_kxr_kernel(const int8_t* __restrict__ X, int64_t R, int64_t K, int64_t ld
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             if (r0 + j >= R) continue;
-            if (kMixed) encode32_store_mixed(lut_s, slot, t[j], planes, R, r0 + j, k0, pitch);
+            if (kMixed) encode32_store_mixed(lut_s, slot, t[j], planes, planes4, plane_stride, r0 + j, k0, pitch);
             else encode32_store<NP>(lut_s, slot, t[j], planes + (r0 + j) * pitch + k0 / 2, plane_stride);
         }
     }
@@ -466,19 +469,19 @@ cudaError_t launch16(awe_layout_t layout, const uint16_t* X, int64_t R, int64_t 
 
 template <int NP, bool kMixed = false, bool kPacked = false>
 cudaError_t launch(awe_layout_t layout, const int8_t* X, int64_t R, int64_t K, int64_t ld, const uint64_t* lut,
-                   uint8_t* planes, int64_t pitch, int64_t plane_stride, int vec_ok, int sm_count,
+                   uint8_t* planes, uint8_t* planes4, int64_t pitch, int64_t plane_stride, int vec_ok, int sm_count,
                    cudaStream_t stream) {
     const int64_t warps_per_block = kEncThreads / 32;
     if (layout == AWE_ROWMAJOR_RxK) {
         const int64_t items = R * ((pitch * 2 + 1023) / 1024);
         const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
         encode_rxk_kernel<NP, kMixed, kPacked><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
-            X, R, K, ld, lut, planes, pitch, plane_stride, vec_ok);
+            X, R, K, ld, lut, planes, planes4, pitch, plane_stride, vec_ok);
     } else {
         const int64_t items = ((pitch * 2 + kKxrK - 1) / kKxrK) * ((R + kKxrRows - 1) / kKxrRows);
         const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
         encode_kxr_kernel<NP, kMixed, kPacked><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
-            X, R, K, ld, lut, planes, pitch, plane_stride, vec_ok);
+            X, R, K, ld, lut, planes, planes4, pitch, plane_stride, vec_ok);
     }
     return cudaGetLastError();
 }
@@ -491,7 +494,14 @@ using namespace awe;
 extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_side_t side, const void* X_dev,
                                    awe_in_dtype_t dt, awe_layout_t layout, int64_t R, int64_t K, int64_t ld,
                                    void* planes_dev, void* stream) {
-    if (!h || !X_dev || !planes_dev || R <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
+    return encode_window(h, enc, modulus, side, X_dev, dt, layout, R, K, ld, PlaneWindow{planes_dev, R, 0}, stream);
+}
+
+awe_status_t awe::encode_window(awe_ctx* h, int enc, int modulus, awe_side_t side, const void* X_dev, awe_in_dtype_t dt,
+                                awe_layout_t layout, int64_t R, int64_t K, int64_t ld, PlaneWindow win, void* stream) {
+    void* planes_dev = const_cast<void*>(win.base);
+    if (!h || !X_dev || !planes_dev || R <= 0 || K <= 0 || win.row0 < 0 || win.row0 + R > win.plane_rows)
+        return AWE_ERR_INVALID_ARG;
     if (side != AWE_SIDE_A && side != AWE_SIDE_B) return AWE_ERR_INVALID_ARG;
     if ((int)dt < 0 || (int)dt > 6) return AWE_ERR_INVALID_ARG;
     if (layout != AWE_ROWMAJOR_RxK && layout != AWE_ROWMAJOR_KxR) return AWE_ERR_INVALID_ARG;
@@ -504,11 +514,15 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
     const uint64_t* lut;
     awe_status_t s = device_lut(h, enc, modulus, side, dt, st, &lut);
     if (s != AWE_OK) return s;
-    const int64_t pitch = plane_pitch_bytes(K), plane_stride = R * pitch;
+    const int64_t pitch = plane_pitch_bytes(K), plane_stride = win.plane_rows * pitch;
     // vector path: 16-byte loads along k (RxK) or 4-byte loads along r (KxR)
     const int64_t align = layout == AWE_ROWMAJOR_RxK ? 16 : 4;
     const int vec_ok = ((uintptr_t)X_dev % align == 0) && (ld % align == 0);
-    uint8_t* P = (uint8_t*)planes_dev;
+    // row 0 of this call inside plane 0; the E4M3 planes of the mixed record (which come first) have rows
+    // twice as long, and its E2M1 plane starts after the two of them
+    const bool mixed = t->bits[0] == 8;
+    uint8_t* P = (uint8_t*)planes_dev + win.row0 * pitch * (mixed ? 2 : 1);
+    uint8_t* P4 = mixed ? (uint8_t*)planes_dev + 4 * plane_stride + win.row0 * pitch : P;
     cudaError_t e;
     if (is_16bit(dt)) {
         if ((uintptr_t)X_dev % 2) return AWE_ERR_ALIGNMENT;
@@ -530,9 +544,9 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
         const int vp = layout == AWE_ROWMAJOR_RxK ? (((uintptr_t)X_dev % 16 == 0) && (ld % 32 == 0))
                                                   : (((uintptr_t)X_dev % 2 == 0) && (ld % 4 == 0));
         switch (t->n_planes) {
-            case 2: e = launch<2, false, true>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vp, h->sm_count, st); break;
-            case 3: e = launch<3, false, true>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vp, h->sm_count, st); break;
-            case 4: e = launch<4, false, true>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vp, h->sm_count, st); break;
+            case 2: e = launch<2, false, true>(layout, X, R, K, ld, lut, P, P4, pitch, plane_stride, vp, h->sm_count, st); break;
+            case 3: e = launch<3, false, true>(layout, X, R, K, ld, lut, P, P4, pitch, plane_stride, vp, h->sm_count, st); break;
+            case 4: e = launch<4, false, true>(layout, X, R, K, ld, lut, P, P4, pitch, plane_stride, vp, h->sm_count, st); break;
             default: return AWE_ERR_UNSUPPORTED;
         }
         if (e != cudaSuccess) return AWE_ERR_CUDA;
@@ -540,17 +554,17 @@ extern "C" awe_status_t awe_encode(awe_handle_t h, int enc, int modulus, awe_sid
         return AWE_OK;
     }
     if (t->bits[0] == 8) {
-        e = launch<3, true>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st);
+        e = launch<3, true>(layout, X, R, K, ld, lut, P, P4, pitch, plane_stride, vec_ok, h->sm_count, st);
         if (e != cudaSuccess) return AWE_ERR_CUDA;
         h->launches += 1;
         return AWE_OK;
     }
     switch (t->n_planes) {
-        case 1: e = launch<1>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st); break;
-        case 2: e = launch<2>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st); break;
-        case 3: e = launch<3>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st); break;
-        case 4: e = launch<4>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st); break;
-        case 6: e = launch<6>(layout, X, R, K, ld, lut, P, pitch, plane_stride, vec_ok, h->sm_count, st); break;
+        case 1: e = launch<1>(layout, X, R, K, ld, lut, P, P4, pitch, plane_stride, vec_ok, h->sm_count, st); break;
+        case 2: e = launch<2>(layout, X, R, K, ld, lut, P, P4, pitch, plane_stride, vec_ok, h->sm_count, st); break;
+        case 3: e = launch<3>(layout, X, R, K, ld, lut, P, P4, pitch, plane_stride, vec_ok, h->sm_count, st); break;
+        case 4: e = launch<4>(layout, X, R, K, ld, lut, P, P4, pitch, plane_stride, vec_ok, h->sm_count, st); break;
+        case 6: e = launch<6>(layout, X, R, K, ld, lut, P, P4, pitch, plane_stride, vec_ok, h->sm_count, st); break;
         default: return AWE_ERR_UNSUPPORTED;
     }
     if (e != cudaSuccess) return AWE_ERR_CUDA;

@@ -591,7 +591,18 @@ using namespace awe;
 extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, const void* planesA_dev,
                                         const void* planesB_dev, int64_t M, int64_t N, int64_t K, void* C_dev,
                                         awe_out_dtype_t out_dt, int64_t ldc, int64_t k_chunk, void* stream) {
+    return gemm_planes_window(h, enc, modulus, PlaneWindow{planesA_dev, M, 0}, PlaneWindow{planesB_dev, N, 0}, M, N, K,
+                              C_dev, out_dt, ldc, k_chunk, stream);
+}
+
+awe_status_t awe::gemm_planes_window(awe_ctx* h, int enc, int modulus, PlaneWindow wa, PlaneWindow wb, int64_t M,
+                                     int64_t N, int64_t K, void* C_dev, awe_out_dtype_t out_dt, int64_t ldc,
+                                     int64_t k_chunk, void* stream) {
+    const void* planesA_dev = wa.base;
+    const void* planesB_dev = wb.base;
     if (!h || !planesA_dev || !planesB_dev || !C_dev || M <= 0 || N <= 0 || K <= 0) return AWE_ERR_INVALID_ARG;
+    if (wa.row0 < 0 || wa.row0 + M > wa.plane_rows || wb.row0 < 0 || wb.row0 + N > wb.plane_rows)
+        return AWE_ERR_INVALID_ARG;
     // 32-bit tile counters and TMA coordinates: at most 2^31 bytes along a plane row and 2^30 tiles
     if (M > (1 << 30) || N > (1 << 30) || K > (1ll << 31)) return AWE_ERR_INVALID_ARG;
     if (((M + 127) / 128) * ((N + 127) / 128) > (1ll << 30)) return AWE_ERR_INVALID_ARG;
@@ -635,16 +646,19 @@ extern "C" awe_status_t awe_gemm_planes(awe_handle_t h, int enc, int modulus, co
     const bool mixed = n8a > 0 || n8b > 0;
     if (mixed && (wide || residue || !use_pairs() || n8a == d.n_planes_a || n8b == d.n_planes_b))
         return AWE_ERR_UNSUPPORTED;
-    const uint8_t* a4 = (const uint8_t*)planesA_dev + (size_t)n8a * M * 2 * pitch;
-    const uint8_t* b4 = (const uint8_t*)planesB_dev + (size_t)n8b * N * 2 * pitch;
+    // row 0 of the window in the first E2M1 plane and in the first E4M3 plane of each side
+    const uint8_t* a4 = (const uint8_t*)planesA_dev + ((size_t)n8a * wa.plane_rows * 2 + (size_t)wa.row0) * pitch;
+    const uint8_t* b4 = (const uint8_t*)planesB_dev + ((size_t)n8b * wb.plane_rows * 2 + (size_t)wb.row0) * pitch;
+    const uint8_t* a8 = (const uint8_t*)planesA_dev + (size_t)wa.row0 * 2 * pitch;
+    const uint8_t* b8 = (const uint8_t*)planesB_dev + (size_t)wb.row0 * 2 * pitch;
     CUtensorMap ma, mb, ma8, mb8;
-    if ((s = make_plane_map(h, a4, M, pitch, d.n_planes_a - n8a, kTileM, &ma)) != AWE_OK) return s;
-    if ((s = make_plane_map(h, b4, N, pitch, d.n_planes_b - n8b, wide ? wide_b_box_rows() : b_box_rows(), &mb)) !=
-        AWE_OK)
+    if ((s = make_plane_map(h, a4, M, pitch, d.n_planes_a - n8a, kTileM, &ma, wa.plane_rows)) != AWE_OK) return s;
+    if ((s = make_plane_map(h, b4, N, pitch, d.n_planes_b - n8b, wide ? wide_b_box_rows() : b_box_rows(), &mb,
+                            wb.plane_rows)) != AWE_OK)
         return s;
     if (mixed) {
-        if ((s = make_plane_map(h, planesA_dev, M, 2 * pitch, n8a, kTileM, &ma8)) != AWE_OK) return s;
-        if ((s = make_plane_map(h, planesB_dev, N, 2 * pitch, n8b, Cfg<true>::kBRows, &mb8)) != AWE_OK) return s;
+        if ((s = make_plane_map(h, a8, M, 2 * pitch, n8a, kTileM, &ma8, wa.plane_rows)) != AWE_OK) return s;
+        if ((s = make_plane_map(h, b8, N, 2 * pitch, n8b, Cfg<true>::kBRows, &mb8, wb.plane_rows)) != AWE_OK) return s;
     }
 
     GemmParams p = {};

@@ -104,6 +104,19 @@ struct awe_ctx {
 };
 
 namespace awe {
+// The stored planes of an operand seen as a window of rows [row0, row0 + R) inside a plane set whose
+// planes are plane_rows rows apart (the whole set when row0 = 0 and plane_rows = R).  Lets the
+// host-buffer path encode an operand chunk by chunk into one plane set and multiply any row range of it.
+struct PlaneWindow {
+    const void* base;    // start of the whole plane set
+    int64_t plane_rows;  // rows per plane of the whole set
+    int64_t row0;        // first row of the window
+};
+awe_status_t encode_window(awe_ctx* h, int enc, int modulus, awe_side_t side, const void* X_dev, awe_in_dtype_t dt,
+                           awe_layout_t layout, int64_t R, int64_t K, int64_t ld, PlaneWindow win, void* stream);
+awe_status_t gemm_planes_window(awe_ctx* h, int enc, int modulus, PlaneWindow a, PlaneWindow b, int64_t M, int64_t N,
+                                int64_t K, void* C_dev, awe_out_dtype_t out_dt, int64_t ldc, int64_t k_chunk,
+                                void* stream);
 // Table arena of a handle: room for both sides of every modulus 2..169 and of every exact
 // encoding in each input container, so that no table ever has to be evicted.
 constexpr int kLutSlots = 512;

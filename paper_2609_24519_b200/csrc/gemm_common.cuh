@@ -169,12 +169,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// planes: n_planes x rows x pitch bytes.  Box: 128 bytes of K x box_rows rows of one plane.
+// planes: n_planes planes of `rows` rows of pitch bytes, plane j starting plane_rows rows after plane
+// j - 1 (plane_rows = 0: the planes are dense, rows apart).  Box: 128 bytes of K x box_rows rows of one plane.
 inline awe_status_t make_plane_map(awe_ctx* h, const void* planes, int64_t rows, int64_t pitch, int n_planes,
-                            int box_rows, CUtensorMap* out) {
+                            int box_rows, CUtensorMap* out, int64_t plane_rows = 0) {
     if (!h->encode_tiled) return AWE_ERR_CUDA;
+    if (plane_rows == 0) plane_rows = rows;
     cuuint64_t dims[3] = {(cuuint64_t)pitch, (cuuint64_t)rows, (cuuint64_t)n_planes};
-    cuuint64_t strides[2] = {(cuuint64_t)pitch, (cuuint64_t)pitch * (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)pitch, (cuuint64_t)pitch * (cuuint64_t)plane_rows};
     cuuint32_t box[3] = {(cuuint32_t)kBlockKBytes, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = ((EncodeTiledFn)h->encode_tiled)(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(planes),

@@ -313,9 +313,9 @@ def test_host_buffer_entry_point_row_chunks_and_column_blocks(enc, out_dt, tdt, 
     b.awe_gemm_exact_host(h, Ah, a_dt, Bh, b.I8, w.M, w.N, w.K, enc, 0, Ch, out_dt, scratch)
     assert b.awe_last_device_status(h) == (0, 0)
     got = Ch.numpy().astype(np.int64)
-    rows = [0, 2047, 2048, 2303, 4095, 4096, 4499]
+    rows = [0, 511, 512, 1023, 1024, 2047, 2048, 2303, 4095, 4096, 4499]      # both sides of every chunk edge
     assert np.array_equal(got[rows], mm.matmul_i64(A[rows], B))
-    cols = [0, 2047, 2048, 4095, 4096, 6143, 6144, 6399]
+    cols = [0, 2047, 2048, 2559, 2560, 3071, 3072, 4095, 4096, 6143, 6144, 6399]
     assert np.array_equal(got[:, cols], mm.matmul_i64(A, np.ascontiguousarray(B[:, cols])))
     # whole matrix against the device-buffer entry point
     assert np.array_equal(got, gu.gpu_gemm_exact(A, B, enc, out_dt, a_dt=a_dt).astype(np.int64))
