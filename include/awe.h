@@ -79,12 +79,17 @@ typedef enum {
                                    -16), 3 products: the Karatsuba-type step on two limbs (Section 6.1;
                                    the weights are not printed: w = v = (1,4), planes a0, a1, a0-a1,
                                    xy = 5 a0b0 + 20 a1b1 - 4 (a0-a1)(b0-b1)).  Inputs AWE_I5_IN_I8.    */
-    AWE_ENC_BF16SIG_8 = 11      /* BF16 significands with sign (width 9, |x| <= 255; the table also
+    AWE_ENC_BF16SIG_8 = 11,     /* BF16 significands with sign (width 9, |x| <= 255; the table also
                                    covers -256), 8 products (count from Section 6.2's table; the record
                                    is not printed): w = v = (4,9,61), planes a0, a1, a2, a0+a1, one
                                    Karatsuba-type step on the pair (a0, a1),
                                    xy = -20 a0b0 + 45 a1b1 + 3721 a2b2 + 36 (a0+a1)(b0+b1)
                                         + 244 (a0b2 + a2b0) + 549 (a1b2 + a2b1).  Inputs AWE_I9_IN_I16. */
+    AWE_ENC_INT8_AWE6_DERIVED = 12 /* the record of AWE_ENC_INT8_AWE6 with only its three limb planes per side
+                                   stored; the planes a_i + a_j of products 4..6 are formed inside the
+                                   product kernel, in shared memory, from the limb tiles (the alternative
+                                   Section 6.1 weighs when it speaks of the cost of producing planes).
+                                   Half the plane bytes, same result; kept as a measured comparison.   */
 } awe_encoding_t;
 
 typedef enum {
@@ -134,6 +139,8 @@ typedef struct {
     int32_t plane_bits_a[AWE_MAX_PLANES]; /* storage width of each stored plane: 4 (E2M1) or 8 (E4M3) */
     int32_t plane_bits_b[AWE_MAX_PLANES];
     int32_t fp8[AWE_MAX_PRODUCTS];  /* 1 if product k multiplies E4M3 planes (an FP8 GEMM), else 0 */
+    int32_t ia2[AWE_MAX_PRODUCTS];  /* -1, or a second stored plane of A: product k multiplies the sum of */
+    int32_t ib2[AWE_MAX_PRODUCTS];  /* planes ia[k] and ia2[k] (ib[k] and ib2[k]), formed in the kernel    */
 } awe_encoding_desc;
 
 /* Create / destroy a handle bound to CUDA device `device`.  awe_create makes that device

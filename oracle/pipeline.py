@@ -59,6 +59,20 @@ def encode_planes(s: Scheme, side: str, X: np.ndarray, lo: int = -128, hi: int =
     return np.ascontiguousarray(np.moveaxis(pl, -1, 0))
 
 
+def encode_limbs(s: Scheme, side: str, X: np.ndarray, lo: int = -128, hi: int = 127) -> np.ndarray:
+    """First loop of Algorithm 1 alone: result[i] is the R x K int8 matrix of limb i (elements of S) with
+    w . limbs = X (congruent mod m for a residue scheme).  The second loop -- forming plane alpha_k as
+    sum_i alpha_k[i] * limb i -- applied to this gives the planes encode_planes returns."""
+    t = encoder_table(s, side)
+    n = len(s.side(side)[0])
+    lut = np.zeros((hi - lo + 1, n), dtype=np.int8)
+    for x in range(lo, hi + 1):
+        lut[x - lo] = t[x % s.modulus if s.modulus else x]
+    Xi = np.asarray(X).astype(np.int64)
+    assert Xi.min(initial=0) >= lo and Xi.max(initial=0) <= hi
+    return np.ascontiguousarray(np.moveaxis(lut[Xi - lo], -1, 0))
+
+
 def pack_e2m1(plane: np.ndarray) -> np.ndarray:
     """Pack an R x K matrix of S values into E2M1 nibbles, two per byte along K, the
     element with the even K index in the low nibble; K is zero-padded to even."""

@@ -25,6 +25,7 @@ ENC_FP16SIG_AWE12 = 8
 ENC_INT8_MIXED_FP8_3 = 9
 ENC_FP8SIG_3 = 10
 ENC_BF16SIG_8 = 11
+ENC_INT8_AWE6_DERIVED = 12
 I8, I4_IN_I8, T2_IN_I8, I16, I4_PACKED, I5_IN_I8, I9_IN_I16 = 0, 1, 2, 3, 4, 5, 6
 C_I32, C_I64, C_RES_I16, C_RES_I32 = 0, 1, 2, 3
 SIDE_A, SIDE_B = 0, 1
@@ -46,7 +47,8 @@ class EncodingDesc(ctypes.Structure):
                 ("c_a", ctypes.c_int32), ("c_b", ctypes.c_int32), ("k_star", ctypes.c_int64),
                 ("a_lo", ctypes.c_int32), ("a_hi", ctypes.c_int32), ("b_lo", ctypes.c_int32),
                 ("b_hi", ctypes.c_int32), ("plane_bits_a", ctypes.c_int32 * MAX_PLANES),
-                ("plane_bits_b", ctypes.c_int32 * MAX_PLANES), ("fp8", ctypes.c_int32 * MAX_PRODUCTS)]
+                ("plane_bits_b", ctypes.c_int32 * MAX_PLANES), ("fp8", ctypes.c_int32 * MAX_PRODUCTS),
+                ("ia2", ctypes.c_int32 * MAX_PRODUCTS), ("ib2", ctypes.c_int32 * MAX_PRODUCTS)]
 
 
 class AweError(RuntimeError):

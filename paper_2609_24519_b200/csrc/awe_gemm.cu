@@ -18,6 +18,12 @@
 // kMixed instantiation: an E4M3 product streams one-byte elements through the same ring and the
 // same descriptors with tcgen05.mma kind::f8f6f4, and its accumulator holds the product itself.
 //
+// The kDerive instantiation stores only the limb planes of a record whose other planes are sums of two
+// limbs (a_i + a_j): for such a product the producer brings the two limb tiles of each side into two
+// consecutive stages, six extra warps add them nibble by nibble (E2M1 codes through a 256-entry table)
+// into the first stage, and the MMAs run on the result; the paper's remark on the cost of producing
+// planes (Section 6.1), measured.
+//
 // 32-bit wrap-around is deliberate: sum_k l_k P_k is computed modulo 2^32, which equals the
 // true D*C whenever |D*C| < 2^31 (checked on the host), although single terms may exceed it.
 //
@@ -50,7 +56,7 @@ struct Cfg {
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kStages = kPair ? AWE_PAIR_STAGES : 4;
     static constexpr int kCtas = kPair ? 2 : 1;
-    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 8 * 4096 + 256;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 8 * 4096 + 1024;
     // mxf4 instruction descriptor: E2M1 x E2M1, both K-major, UE8M0 scales, dense K = 64
     static constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | (1u << 23) |
                                        ((uint32_t)((kTileM * kCtas) >> 4) << 24);
@@ -72,8 +78,10 @@ struct Shared {
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint64_t overlap_free;
+    uint64_t formed[kMaxStages];  // kDerive: the stage's tiles are complete (sums formed), both CTAs
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
+    uint8_t add_lo[256], add_hi[256];  // kDerive: E2M1 code of x + y for codes (x, y), in the low / high nibble
 };
 
 
@@ -107,6 +115,28 @@ __device__ __forceinline__ float mod_symmetric(float x, float m, float inv_m, fl
     r = r > hi ? r - m : r;
     r = r < lo ? r + m : r;
     return r;
+}
+
+// E2M1 code <-> doubled integer (Section 3.1): sign, two exponent bits, one mantissa bit.
+__device__ __forceinline__ int e2m1_value(int code) {
+    const int e = (code >> 1) & 3, m = code & 1;
+    const int v = e ? (2 + m) << (e - 1) : m;
+    return (code & 8) ? -v : v;
+}
+__device__ __forceinline__ int e2m1_code(int v) {
+    const int a = v < 0 ? -v : v;
+    const int mag = a <= 4 ? a : (a == 6 ? 5 : (a == 8 ? 6 : (a == 12 ? 7 : 0)));
+    return mag | ((v < 0 && mag) ? 8 : 0);
+}
+// Nibble-wise sum of two words of eight E2M1 codes (every sum lies in S by construction of the record).
+__device__ __forceinline__ uint32_t add_e2m1x8(uint32_t x, uint32_t y, const uint8_t* lo, const uint8_t* hi) {
+    const uint32_t il = (x & 0x0F0F0F0Fu) | ((y << 4) & 0xF0F0F0F0u);
+    const uint32_t ih = ((x >> 4) & 0x0F0F0F0Fu) | (y & 0xF0F0F0F0u);
+    uint32_t z = 0;
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+        z |= (uint32_t)(lo[(il >> (8 * b)) & 255u] | hi[(ih >> (8 * b)) & 255u]) << (8 * b);
+    return z;
 }
 
 struct EpiMath {
@@ -157,12 +187,14 @@ __device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128]
 // elements per 128-byte K block, kind::f8f6f4 without block scales, accumulator = the product
 // itself); the others are E2M1 products as above.  Pair variant only.
 // kGrouped: the reconstruction is a weighted sum of cells whose own sums fit 32 bits (GemmParams::group_*).
-template <bool kPair, bool kMixed, bool kGrouped>
-__global__ void __launch_bounds__(kThreads, 1)
+// kDerive: products with ia2[k] >= 0 multiply sum planes formed in shared memory (pair variant only).
+template <bool kPair, bool kMixed, bool kGrouped, bool kDerive = false>
+__global__ void __launch_bounds__(kDerive ? kThreadsDerive : kThreads, 1)
 awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a8, const __grid_constant__ CUtensorMap map_b8,
                 const __grid_constant__ GemmParams p) {
     static_assert(kPair || !kMixed, "mixed-format records run on CTA pairs");
+    static_assert(!kDerive || (kPair && !kMixed && !kGrouped), "sum planes are formed in the plain pair variant only");
     using C = Cfg<kPair>;
     constexpr int kStages = C::kStages;
     constexpr int kStageBytes = C::kStageBytes;
@@ -188,6 +220,8 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             ptx::mbar_init(ptx::smem_u32(&sh->acc_empty[b]), kEpiWarps * C::kCtas);
         }
         ptx::mbar_init(ptx::smem_u32(&sh->overlap_free), (kEpiWarps / 2) * C::kCtas);
+        if (kDerive)
+            for (int s = 0; s < kStages; ++s) ptx::mbar_init(ptx::smem_u32(&sh->formed[s]), kFormerWarps * C::kCtas);
         sh->abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&map_a);
@@ -205,6 +239,12 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), kTmemCols);
             ptx::tmem_relinquish();
         }
+    }
+    if (kDerive && threadIdx.x >= 256) {
+        const int idx = (int)threadIdx.x - 256;  // codes (x, y) = (idx & 15, idx >> 4)
+        const int code = e2m1_code(e2m1_value(idx & 15) + e2m1_value(idx >> 4));
+        sh->add_lo[idx] = (uint8_t)code;
+        sh->add_hi[idx] = (uint8_t)(code << 4);
     }
     ptx::tc_fence_before();
     __syncthreads();
@@ -255,7 +295,23 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         const uint32_t bar = ptx::smem_u32(&sh->full[s]);
                         const uint32_t a_dst = tiles_base + s * kStageBytes;
                         const int x = (kb_first + kb) * kBlockKBytes;
-                        if (kPair) {
+                        if (kDerive) {
+                            // every CTA counts its own bytes on its own barrier (its forming warps wait there);
+                            // a product of sum planes fills a second stage with the tiles to be added
+                            ptx::mbar_arrive_expect_tx(bar, kStageBytes);
+                            ptx::tma_load_3d(a_dst, &map_a, bar, x, row_a, p.ia[k]);
+                            ptx::tma_load_3d(a_dst + kABytes, &map_b, bar, x, row_b, p.ib[k]);
+                            if (p.ia2[k] >= 0) {
+                                ++it;
+                                const uint32_t s2 = it % kStages, ph2 = (it / kStages) & 1u;
+                                if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->empty[s2]), ph2 ^ 1u, p.status, 6))) break;
+                                const uint32_t bar2 = ptx::smem_u32(&sh->full[s2]);
+                                const uint32_t dst2 = tiles_base + s2 * kStageBytes;
+                                ptx::mbar_arrive_expect_tx(bar2, kStageBytes);
+                                ptx::tma_load_3d(dst2, &map_a, bar2, x, row_a, p.ia2[k]);
+                                ptx::tma_load_3d(dst2 + kABytes, &map_b, bar2, x, row_b, p.ib2[k]);
+                            }
+                        } else if (kPair) {
                             // both CTAs report their bytes to CTA 0's barrier, which expects the sum
                             if (rank == 0) ptx::mbar_arrive_expect_tx(bar, 2 * kStageBytes);
                             const uint32_t bar0 = ptx::map_to_cta(bar, 0);
@@ -285,11 +341,18 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // One accumulation segment: K blocks [kb0, kb_end) into the accumulator at acc_col.  The
             // operand format is a compile-time constant of the loop: a per-instruction test of a
             // run-time flag here slowed every instruction of either format by half.
+            bool sum_planes = false;  // kDerive: the current product multiplies sums of two stored planes
             auto issue_segment = [&](auto is_f8, int kb0, int kb_end, uint32_t acc_col, bool carry) {
                 constexpr bool kF8 = decltype(is_f8)::value;
                 for (int kb = kb0; kb < kb_end; ++kb, ++it) {
                     const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
-                    if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->full[s]), ph, p.status, 3))) break;
+                    if (kDerive) {
+                        // the forming warps of both CTAs have passed (and, for sum planes, rewritten) the stage
+                        if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->formed[s]), ph, p.status, 7))) break;
+                        ptx::fence_acq_rel_cluster();
+                    } else if (!(ok = bounded_wait(sh, ptx::smem_u32(&sh->full[s]), ph, p.status, 3))) {
+                        break;
+                    }
                     ptx::tc_fence_after();
                     const uint32_t a_addr = tiles_base + s * kStageBytes;
                     const uint64_t a_desc = ptx::smem_desc_k_sw128(a_addr);
@@ -310,12 +373,17 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     // frees the stage in both CTAs of a pair
                     if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->empty[s]), 3);
                     else ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));
+                    if (kDerive && sum_planes) {  // the stage that held the tiles added in goes back as well
+                        ++it;
+                        ptx::mma_commit_pair(ptx::smem_u32(&sh->empty[it % kStages]), 3);
+                    }
                 }
             };
             for (int t = worker, tile_iter = 0; t < num_tiles && ok; t += num_workers, ++tile_iter) {
                 for (int kk = 0; kk < p.r && ok; ++kk) {
                     const int k = product_at(kk, tile_iter, p.r);
                     const bool f8 = kMixed && p.fp8[k];
+                    if (kDerive) sum_planes = p.ia2[k] >= 0;
                     const int nkb = f8 ? p.num_kblocks8 : p.num_kblocks;
                     const int ckb = f8 ? p.chunk_kblocks8 : p.chunk_kblocks;
                     const int nchunks = f8 ? chunks8 : chunks;
@@ -348,6 +416,47 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             ++drains;
                         }
                     }
+                }
+            }
+        }
+    } else if (kDerive && warp >= 2 + kEpiWarps) {
+        // -------------------------------------------------------------------- forming warps (kDerive)
+        // They follow the producer's sequence of stages.  A stage of a plain product is only passed on;
+        // for a product of sum planes the tiles of the following stage are added, 16 bytes at a time,
+        // into the stage the MMAs will read (both tiles of a side were written by TMA with the same
+        // swizzle, so the sum is elementwise on equal offsets).
+        const int ftid = (int)threadIdx.x - 32 * (2 + kEpiWarps);
+        uint32_t formed_bar[kMaxStages];
+        for (int s = 0; s < kStages; ++s) formed_bar[s] = ptx::map_to_cta(ptx::smem_u32(&sh->formed[s]), 0);
+        uint32_t it = 0;
+        bool ok = true;
+        for (int t = worker, tile_iter = 0; t < num_tiles && ok; t += num_workers, ++tile_iter) {
+            for (int kk = 0; kk < p.r && ok; ++kk) {
+                const int k = product_at(kk, tile_iter, p.r);
+                const bool sum = p.ia2[k] >= 0;
+                for (int kb = 0; kb < p.num_kblocks && ok; ++kb, ++it) {
+                    const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+                    ok = __all_sync(0xffffffffu, bounded_wait(sh, ptx::smem_u32(&sh->full[s]), ph, p.status, 8));
+                    if (!ok) break;
+                    if (sum) {
+                        ++it;
+                        const uint32_t s2 = it % kStages, ph2 = (it / kStages) & 1u;
+                        ok = __all_sync(0xffffffffu, bounded_wait(sh, ptx::smem_u32(&sh->full[s2]), ph2, p.status, 9));
+                        if (!ok) break;
+                        uint4* dst = reinterpret_cast<uint4*>(smem_raw + (tiles_base - raw) + (size_t)s * kStageBytes);
+                        const uint4* src =
+                            reinterpret_cast<const uint4*>(smem_raw + (tiles_base - raw) + (size_t)s2 * kStageBytes);
+                        for (int c = ftid; c < kStageBytes / 16; c += 32 * kFormerWarps) {
+                            const uint4 x = dst[c], y = src[c];
+                            dst[c] = make_uint4(add_e2m1x8(x.x, y.x, sh->add_lo, sh->add_hi),
+                                                add_e2m1x8(x.y, y.y, sh->add_lo, sh->add_hi),
+                                                add_e2m1x8(x.z, y.z, sh->add_lo, sh->add_hi),
+                                                add_e2m1x8(x.w, y.w, sh->add_lo, sh->add_hi));
+                        }
+                        ptx::fence_proxy_async();  // the MMAs read these bytes through the async proxy
+                        release(formed_bar[s2], lane, true);  // keeps the unused barrier's phase in step
+                    }
+                    release(formed_bar[s], lane, true);
                 }
             }
         }
@@ -528,13 +637,13 @@ bool use_pairs() {
     return v;
 }
 
-template <bool kPair, bool kMixed, bool kGrouped = false>
+template <bool kPair, bool kMixed, bool kGrouped = false, bool kDerive = false>
 awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ma8,
                             const CUtensorMap& mb8, GemmParams& p, cudaStream_t st) {
     using C = Cfg<kPair>;
-    bool& attr_set = h->smem_attr_set[kGrouped ? 4 : (kMixed ? 3 : (kPair ? 0 : 1))];
+    bool& attr_set = h->smem_attr_set[kDerive ? 5 : (kGrouped ? 4 : (kMixed ? 3 : (kPair ? 0 : 1)))];
     if (!attr_set) {
-        if (cudaFuncSetAttribute(awe_gemm_kernel<kPair, kMixed, kGrouped>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(awe_gemm_kernel<kPair, kMixed, kGrouped, kDerive>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)C::kSmemBytes) != cudaSuccess)
             return AWE_ERR_CUDA;
         attr_set = true;
@@ -546,7 +655,7 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
     const int workers = std::min(p.tiles_m * p.tiles_n, h->sm_count / C::kCtas);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(workers * C::kCtas));
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(kDerive ? kThreadsDerive : kThreads);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -556,7 +665,7 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair, kMixed, kGrouped>, ma, mb, ma8, mb8, p);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair, kMixed, kGrouped, kDerive>, ma, mb, ma8, mb8, p);
     if (err != cudaSuccess) {
         if (getenv("AWE_DEBUG")) fprintf(stderr, "awe: GEMM launch failed: %s\n", cudaGetErrorString(err));
         return AWE_ERR_CUDA;
@@ -567,6 +676,9 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
 
 awe_status_t launch_gemm(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmParams& p, cudaStream_t st) {
     if (p.grouped) return launch_variant<true, false, true>(h, ma, mb, ma, mb, p, st);
+    bool derive = false;
+    for (int k = 0; k < p.r; ++k) derive = derive || p.ia2[k] >= 0;
+    if (derive) return launch_variant<true, false, false, true>(h, ma, mb, ma, mb, p, st);
     return use_pairs() ? launch_variant<true, false>(h, ma, mb, ma, mb, p, st)
                        : launch_variant<false, false>(h, ma, mb, ma, mb, p, st);
 }
@@ -671,6 +783,14 @@ awe_status_t awe::gemm_planes_window(awe_ctx* h, int enc, int modulus, PlaneWind
         p.ib[k] = d.fp8[k] ? d.ib[k] : d.ib[k] - n8b;
         p.ell[k] = d.ell[k];
     }
+    bool derive = false;
+    for (int k = 0; k < AWE_MAX_PRODUCTS; ++k) {
+        p.ia2[k] = k < d.r ? d.ia2[k] : -1;
+        p.ib2[k] = k < d.r ? d.ib2[k] : -1;
+        if ((p.ia2[k] >= 0) != (p.ib2[k] >= 0)) return AWE_ERR_UNSUPPORTED;  // sums are formed on both sides or on none
+        derive = derive || p.ia2[k] >= 0;
+    }
+    if (derive && (wide || grouped || mixed || residue || !use_pairs())) return AWE_ERR_UNSUPPORTED;
     p.log2D = d.log2D;
     p.modulus = d.modulus;
     p.out_mode = (int)out_dt;
@@ -747,6 +867,8 @@ awe_status_t awe::gemm_planes_window(awe_ctx* h, int enc, int modulus, PlaneWind
                 q.ib[k] = p.ib[ord[k]];
                 q.ell[k] = p.ell[ord[k]];
                 q.fp8[k] = p.fp8[ord[k]];
+                q.ia2[k] = p.ia2[ord[k]];
+                q.ib2[k] = p.ib2[ord[k]];
                 q.group_id[k] = p.group_id[ord[k]];
                 q.group_scale[k] = p.group_scale[ord[k]];
                 q.set_id[k] = set_of[k];
@@ -798,6 +920,7 @@ extern "C" awe_status_t awe_fp4_product_raw(awe_handle_t h, const void* planeX_d
     p.N = (int)N;
     p.r = 1;
     p.ell[0] = 1;
+    for (int k = 0; k < AWE_MAX_PRODUCTS; ++k) p.ia2[k] = p.ib2[k] = -1;
     p.out_mode = OUT_RAW_F32;
     p.C = P_dev;
     p.ldc = ldp;
@@ -827,6 +950,7 @@ extern "C" awe_status_t awe_fp8_product_raw(awe_handle_t h, const void* planeX_d
     p.N = (int)N;
     p.r = 1;
     p.ell[0] = 1;
+    for (int k = 0; k < AWE_MAX_PRODUCTS; ++k) p.ia2[k] = p.ib2[k] = -1;
     p.fp8[0] = 1;
     p.out_mode = OUT_RAW_F32;
     p.C = P_dev;

@@ -30,6 +30,8 @@ struct SideTable {
     int n_planes = 0;
     int planes[AWE_MAX_PLANES][kMaxLimbs] = {{0}};
     int index_of_product[AWE_MAX_PRODUCTS] = {0};
+    int index2_of_product[AWE_MAX_PRODUCTS];  // second stored plane whose sum with the first is multiplied, or -1
+    SideTable() { for (int& x : index2_of_product) x = -1; }
     int bits[AWE_MAX_PLANES] = {4, 4, 4, 4, 4, 4, 4, 4};  // storage width: 4 = E2M1 nibble, 8 = E4M3 byte
     int c = 0;       // largest |plane value| over the input range
     int entries = 0; // 256 (index: raw byte) or 4096 (index: low 12 bits of a 16-bit element)
@@ -100,7 +102,7 @@ struct awe_ctx {
     cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_done = nullptr;
     cudaEvent_t ev_a[kMaxHostChunks] = {nullptr}, ev_bcol[kMaxHostColBlocks] = {nullptr};
     cudaEvent_t ev_c[kMaxHostChunks * kMaxHostColBlocks] = {nullptr};
-    bool smem_attr_set[5] = {false, false, false, false, false};  // dynamic shared-memory limit raised (per kernel, this device)
+    bool smem_attr_set[6] = {false, false, false, false, false, false};  // dynamic shared-memory limit raised (per kernel, this device)
 };
 
 namespace awe {

@@ -458,6 +458,7 @@ bool get_scheme(int enc, int modulus, Scheme* out) {
     if (enc != AWE_ENC_MOD_M && modulus != 0) return false;
     switch (enc) {
         case AWE_ENC_INT8_AWE6:
+        case AWE_ENC_INT8_AWE6_DERIVED:
             s = make_awe6(29, 37, {-65, -261, 259, 29, 37, 1073});
             ok = true;
             break;
@@ -513,6 +514,58 @@ bool get_side_table(int enc, int modulus, awe_side_t side, awe_in_dtype_t dt, co
     dt = table_dtype(dt);
     Scheme s;
     if (!get_scheme(enc, modulus, &s)) return false;
+    if (enc == AWE_ENC_INT8_AWE6_DERIVED) {
+        // The tuples are those of the full record (all six plane values must lie in S); only the limb
+        // planes are stored, and a product of two sum planes names the two limb planes it adds.
+        const SideTable* full;
+        if (!get_side_table(AWE_ENC_INT8_AWE6, modulus, side, dt, &full)) return false;
+        std::lock_guard<std::mutex> lock(g_mu);
+        auto key = std::make_tuple(enc, modulus, (int)side, (int)dt);
+        auto it = g_tables.find(key);
+        if (it == g_tables.end()) {
+            SideTable t = *full;
+            const int n = side == AWE_SIDE_A ? s.p : s.q;
+            t.n_planes = n;
+            for (int j = 0; j < AWE_MAX_PLANES; ++j)
+                for (int i = 0; i < kMaxLimbs; ++i) t.planes[j][i] = (j < n && i == j) ? 1 : 0;
+            for (int k = 0; k < s.r; ++k) {
+                const int* pl = side == AWE_SIDE_A ? s.alpha[k] : s.beta[k];
+                int first = -1, second = -1;
+                for (int i = 0; i < n; ++i) {
+                    if (pl[i] == 0) continue;
+                    if (pl[i] != 1 || second >= 0) return false;  // only sums of two limbs are formed in the kernel
+                    (first < 0 ? first : second) = i;
+                }
+                if (first < 0) return false;
+                t.index_of_product[k] = first;
+                t.index2_of_product[k] = second;
+            }
+            for (int b = 0; b < t.entries; ++b) {
+                uint64_t word = 0;
+                for (int j = 0; j < AWE_MAX_PLANES; ++j) {
+                    int8_t& v = t.value[(size_t)b * AWE_MAX_PLANES + j];
+                    if (j >= n) {
+                        v = 0;
+                        continue;
+                    }
+                    // limb j is the value of the full record's plane with the unit vector e_j
+                    int src = -1;
+                    for (int q = 0; q < full->n_planes && src < 0; ++q) {
+                        bool unit = true;
+                        for (int i = 0; i < n; ++i) unit = unit && full->planes[q][i] == (i == j ? 1 : 0);
+                        if (unit) src = q;
+                    }
+                    if (src < 0) return false;
+                    v = full->value[(size_t)b * AWE_MAX_PLANES + src];
+                    word |= (uint64_t)e2m1_code_of(v) << (8 * j);
+                }
+                t.lut[b] = word;
+            }
+            it = g_tables.emplace(key, t).first;
+        }
+        *out = &it->second;
+        return true;
+    }
     std::lock_guard<std::mutex> lock(g_mu);
     auto key = std::make_tuple(enc, modulus, (int)side, (int)dt);
     auto it = g_tables.find(key);
@@ -616,7 +669,10 @@ extern "C" awe_status_t awe_encoding_info(int enc, int modulus, awe_encoding_des
         out->ia[k] = ta->index_of_product[k];
         out->ib[k] = tb->index_of_product[k];
         out->ell[k] = s.ell[k];
+        out->ia2[k] = ta->index2_of_product[k];
+        out->ib2[k] = tb->index2_of_product[k];
     }
+    for (int k = s.r; k < AWE_MAX_PRODUCTS; ++k) out->ia2[k] = out->ib2[k] = -1;
     out->log2D = s.log2D;
     out->modulus = s.modulus;
     out->c_a = ta->c;

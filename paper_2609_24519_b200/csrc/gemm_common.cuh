@@ -15,6 +15,9 @@ constexpr int kABytes = kTileM * kBlockKBytes;  // 16 KB
 
 constexpr int kThreads = 320;
 constexpr int kEpiWarps = 8;
+// The variant that forms sum planes in shared memory adds six warps for that work (warps 10..15).
+constexpr int kThreadsDerive = 512;
+constexpr int kFormerWarps = 6;
 constexpr int kStageWarpBytes = 4096;  // 32 rows x 128 bytes per epilogue warp for the write-out
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSfaCol = 480;  // 16 columns of constant scale bytes each for A and B
@@ -50,6 +53,9 @@ struct GemmParams {
     int group_id[AWE_MAX_PRODUCTS], group_scale[AWE_MAX_PRODUCTS];
     int fp8[AWE_MAX_PRODUCTS];
     int kblock0_8, num_kblocks8, chunk_kblocks8;
+    // Sum planes formed in the kernel: product k multiplies (plane ia[k] + plane ia2[k]) of A by
+    // (plane ib[k] + plane ib2[k]) of B when ia2[k] >= 0 (then ib2[k] >= 0 too); -1 otherwise.
+    int ia2[AWE_MAX_PRODUCTS], ib2[AWE_MAX_PRODUCTS];
 };
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s

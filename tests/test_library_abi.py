@@ -69,6 +69,23 @@ def test_records_match_the_paper_and_the_oracle(b):
     assert (d.c_a, d.c_b, d.k_star) == (3, 8, 699050)
 
 
+def test_record_with_sum_planes_formed_in_the_kernel(b):
+    """AWE_ENC_INT8_AWE6_DERIVED is the 6-product record with only its limb planes stored: same
+    coefficients, three planes per side, products 4..6 name the two limb planes they add, and the table
+    holds the limbs of the oracle's decomposition (whose tuples keep all six plane values in S)."""
+    d6, dd = b.awe_encoding_info(b.ENC_INT8_AWE6), b.awe_encoding_info(b.ENC_INT8_AWE6_DERIVED)
+    assert dd.r == 6 and list(dd.ell)[:6] == list(d6.ell)[:6] and (dd.n_planes_a, dd.n_planes_b) == (3, 3)
+    assert (dd.c_a, dd.c_b, dd.k_star) == (d6.c_a, d6.c_b, d6.k_star)
+    assert list(dd.ia)[:6] == [0, 1, 2, 0, 0, 1] and list(dd.ia2)[:6] == [-1, -1, -1, 1, 2, 2]
+    assert list(dd.ib)[:6] == list(dd.ia)[:6] and list(dd.ib2)[:6] == list(dd.ia2)[:6]
+    assert list(d6.ia2)[:6] == [-1] * 6
+    X = np.arange(-128, 128, dtype=np.int8).reshape(1, 256)
+    for side, name in ((b.SIDE_A, "A"), (b.SIDE_B, "B")):
+        lut = b.awe_encoding_lut(b.ENC_INT8_AWE6_DERIVED, 0, side)
+        assert np.array_equal(lut[np.arange(-128, 128) & 0xFF].T, pl.encode_limbs(sc.AWE6, name, X)[:, 0, :])
+    assert b.awe_planes_bytes(b.ENC_INT8_AWE6_DERIVED, 0, b.SIDE_A, 100, 300) == 3 * 100 * 256
+
+
 def test_tables_match_the_oracle_tables(b):
     idx = np.arange(-128, 128) & 0xFF
     for enc, s in ((b.ENC_INT8_AWE6, sc.AWE6), (b.ENC_INT8_AWE6_ALT, sc.AWE6_ALT), (b.ENC_INT8_BASE13_9, sc.BASE13_9)):

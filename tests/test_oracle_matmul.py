@@ -132,3 +132,21 @@ def test_workload_generators():
     assert A.min() >= -4 and A.max() <= 3
     A2, _ = wl.make_inputs(wl.small("t", 64, 64, 64, "residue", "residue", modulus=8))
     assert np.array_equal(A, A2)
+
+
+def test_limbs_and_plane_formation_are_the_two_loops_of_algorithm1():
+    """First loop (limbs with w . a = x, every limb in S) and second loop (plane alpha_k = sum of limbs)
+    taken apart: together they give the stored planes, for every int8 value."""
+    X = np.arange(-128, 128, dtype=np.int8).reshape(1, 256)
+    for s in (sc.AWE6, sc.AWE6_ALT, sc.BASE13_9):
+        for side in ("A", "B"):
+            limbs = pl.encode_limbs(s, side, X).astype(np.int64)
+            w, _ = s.side(side)
+            assert set(np.unique(limbs)) <= sc.S_SET
+            assert np.array_equal(sum(int(w[i]) * limbs[i] for i in range(len(w))), X.astype(np.int64))
+            planes = pl.encode_planes(s, side, X).astype(np.int64)
+            for j, alpha in enumerate(s.stored_planes(side)):
+                assert np.array_equal(sum(int(alpha[i]) * limbs[i] for i in range(len(w))), planes[j])
+    # the 6-product record stores the three limbs first, then the three pairwise sums
+    assert list(sc.AWE6.stored_planes("A")[:3]) == [(1, 0, 0), (0, 1, 0), (0, 0, 1)]
+    assert list(sc.AWE6.stored_planes("A")[3:]) == [(1, 1, 0), (1, 0, 1), (0, 1, 1)]
