@@ -188,9 +188,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--size", type=int, default=8192, help="M = N = K of the headline workload")
-    ap.add_argument("--encoding", default="awe6", choices=["awe6", "awe6_alt", "base13", "mixed"],
+    ap.add_argument("--encoding", default="awe6", choices=["awe6", "awe6_alt", "base13", "mixed", "derived"],
                     help="INT8xINT8 record of the timed step (the headline metric is awe6)")
     ap.add_argument("--no-extras", action="store_true", help="skip the context measurements")
+    ap.add_argument("--context", default="all",
+                    help="comma list of context measurements to run: base13, mixed, derived, int8, configs, ceiling, "
+                         "reconstruct (default: all)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -226,7 +229,8 @@ def main():
     h = b.awe_create(local_rank)
     enc, enc_name = {"awe6": (b.ENC_INT8_AWE6, "int8_awe6"), "awe6_alt": (b.ENC_INT8_AWE6_ALT, "int8_awe6_alt"),
                      "base13": (b.ENC_INT8_BASE13_9, "int8_base13_9"),
-                     "mixed": (b.ENC_INT8_MIXED_FP8_3, "int8_mixed_2fp8_1fp4")}[args.encoding]
+                     "mixed": (b.ENC_INT8_MIXED_FP8_3, "int8_mixed_2fp8_1fp4"),
+                     "derived": (b.ENC_INT8_AWE6_DERIVED, "int8_awe6_sum_planes_formed_in_kernel")}[args.encoding]
     M, N, K = w.M, w.N, w.K
     A, B = wl.make_inputs(w)
     dA, dB = torch.from_numpy(A).to(dev), torch.from_numpy(B).to(dev)
@@ -383,70 +387,104 @@ def main():
                                     "frac_of_write_bandwidth": enc_write_gbs / fill_gbs})
     del fill_buf
 
+    def want(name):
+        return args.context == "all" or name in args.context.split(",")
+
     if rank == 0 and not args.no_extras:
         ctx = {}
-        # prior-work 9-GEMM base-13 scheme through the same kernels, same inputs
-        enc9 = b.ENC_INT8_BASE13_9
-        ws9 = torch.empty(b.awe_workspace_bytes(enc9, 0, M, N, K), dtype=torch.uint8, device=dev)
-        C9 = torch.empty_like(C)
-        for _ in range(2):
-            b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, enc9, 0, C9, b.C_I32, ws9)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(5):
-            b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, enc9, 0, C9, b.C_I32, ws9)
-        e1.record()
-        torch.cuda.synchronize()
-        ctx["base13_9gemm_TOPS"] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
-        ctx["base13_equals_awe6"] = bool(torch.equal(C9, C))
-        parity_ok = parity_ok and ctx["base13_equals_awe6"]
-        del ws9, C9
-        # mixed 2 x FP8 + 1 x FP4 construction (Appendix A) on the same inputs: whole call and its product kernel
-        encm = b.ENC_INT8_MIXED_FP8_3
-        wsm = torch.empty(b.awe_workspace_bytes(encm, 0, M, N, K), dtype=torch.uint8, device=dev)
-        Cm = torch.empty_like(C)
-        for _ in range(3):
-            b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, encm, 0, Cm, b.C_I32, wsm)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(10):
-            b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, encm, 0, Cm, b.C_I32, wsm)
-        e1.record()
-        torch.cuda.synchronize()
-        ctx["mixed_2fp8_1fp4_TOPS"] = ops / (e0.elapsed_time(e1) / 10 * 1e-3) / 1e12
-        nAm = b.awe_planes_bytes(encm, 0, b.SIDE_A, M, K)
-        pam, pbm = wsm[:nAm], wsm[(nAm + 255) // 256 * 256:]
-        e0.record()
-        for _ in range(10):
-            b.awe_gemm_planes(h, encm, 0, pam, pbm, M, N, K, Cm, b.C_I32, N, 0)
-        e1.record()
-        torch.cuda.synchronize()
-        ctx["mixed_2fp8_1fp4_products_ms"] = e0.elapsed_time(e1) / 10
-        ctx["mixed_sm_mhz"] = b.awe_last_gemm_clock_mhz(h)
-        ctx["mixed_equals_awe6"] = bool(torch.equal(Cm, C))
-        parity_ok = parity_ok and ctx["mixed_equals_awe6"]
-        del wsm, Cm, pam, pbm
-        # INT8 tensor-core GEMM of the same product (library reference point)
-        try:
+        if want("base13"):
+            # prior-work 9-GEMM base-13 scheme through the same kernels, same inputs
+            enc9 = b.ENC_INT8_BASE13_9
+            ws9 = torch.empty(b.awe_workspace_bytes(enc9, 0, M, N, K), dtype=torch.uint8, device=dev)
+            C9 = torch.empty_like(C)
             for _ in range(2):
-                Ci = torch._int_mm(dA, dB)
+                b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, enc9, 0, C9, b.C_I32, ws9)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
             e0.record()
             for _ in range(5):
-                Ci = torch._int_mm(dA, dB)
+                b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, enc9, 0, C9, b.C_I32, ws9)
             e1.record()
             torch.cuda.synchronize()
-            ctx["int8_tensor_core_gemm_TOPS"] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
-            ctx["int8_gemm_equals_awe6"] = bool(torch.equal(Ci, C))
-            parity_ok = parity_ok and ctx["int8_gemm_equals_awe6"]
-            del Ci
-        except Exception as ex:  # library reference point only
-            ctx["int8_tensor_core_gemm_TOPS"] = None
-            ctx["int8_gemm_error"] = str(ex)[:100]
+            ctx["base13_9gemm_TOPS"] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
+            ctx["base13_equals_awe6"] = bool(torch.equal(C9, C))
+            parity_ok = parity_ok and ctx["base13_equals_awe6"]
+            del ws9, C9
+        if want("mixed"):
+            # mixed 2 x FP8 + 1 x FP4 construction (Appendix A) on the same inputs: whole call and its product kernel
+            encm = b.ENC_INT8_MIXED_FP8_3
+            wsm = torch.empty(b.awe_workspace_bytes(encm, 0, M, N, K), dtype=torch.uint8, device=dev)
+            Cm = torch.empty_like(C)
+            for _ in range(3):
+                b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, encm, 0, Cm, b.C_I32, wsm)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(10):
+                b.awe_gemm_exact(h, dA, b.I8, dB, b.I8, M, N, K, encm, 0, Cm, b.C_I32, wsm)
+            e1.record()
+            torch.cuda.synchronize()
+            ctx["mixed_2fp8_1fp4_TOPS"] = ops / (e0.elapsed_time(e1) / 10 * 1e-3) / 1e12
+            nAm = b.awe_planes_bytes(encm, 0, b.SIDE_A, M, K)
+            pam, pbm = wsm[:nAm], wsm[(nAm + 255) // 256 * 256:]
+            e0.record()
+            for _ in range(10):
+                b.awe_gemm_planes(h, encm, 0, pam, pbm, M, N, K, Cm, b.C_I32, N, 0)
+            e1.record()
+            torch.cuda.synchronize()
+            ctx["mixed_2fp8_1fp4_products_ms"] = e0.elapsed_time(e1) / 10
+            ctx["mixed_sm_mhz"] = b.awe_last_gemm_clock_mhz(h)
+            ctx["mixed_equals_awe6"] = bool(torch.equal(Cm, C))
+            parity_ok = parity_ok and ctx["mixed_equals_awe6"]
+            del wsm, Cm, pam, pbm
+        if want("derived") and args.encoding != "derived":
+            # the same record with its sum planes formed inside the product kernel (Section 6.1's alternative)
+            encd = b.ENC_INT8_AWE6_DERIVED
+            wsd = torch.empty(b.awe_workspace_bytes(encd, 0, M, N, K), dtype=torch.uint8, device=dev)
+            Cd = torch.empty_like(C)
+            nAd = b.awe_planes_bytes(encd, 0, b.SIDE_A, M, K)
+            pad, pbd = wsd[:nAd], wsd[(nAd + 255) // 256 * 256:]
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            for it_ in range(4):            # the first pass warms up, the last three are timed
+                if it_ == 1:
+                    torch.cuda.synchronize()
+                    enc_d, prod_d = [], []
+                e0.record()
+                b.awe_encode(h, encd, 0, b.SIDE_A, dA, b.I8, b.ROWMAJOR_RxK, M, K, K, pad)
+                b.awe_encode(h, encd, 0, b.SIDE_B, dB, b.I8, b.ROWMAJOR_KxR, N, K, N, pbd)
+                e1.record()
+                b.awe_gemm_planes(h, encd, 0, pad, pbd, M, N, K, Cd, b.C_I32, N, 0)
+                e2.record()
+                torch.cuda.synchronize()
+                if it_ >= 1:
+                    enc_d.append(e0.elapsed_time(e1))
+                    prod_d.append(e1.elapsed_time(e2))
+            ctx["sum_planes_formed_in_kernel"] = {
+                "encode_a_plus_b_ms": statistics.mean(enc_d), "products_ms": statistics.mean(prod_d),
+                "TOPS": ops / ((statistics.mean(enc_d) + statistics.mean(prod_d)) * 1e-3) / 1e12,
+                "plane_bytes": int(b.awe_workspace_bytes(encd, 0, M, N, K)), "equals_awe6": bool(torch.equal(Cd, C))}
+            parity_ok = parity_ok and ctx["sum_planes_formed_in_kernel"]["equals_awe6"]
+            del wsd, Cd, pad, pbd
+        if want("int8"):
+            # INT8 tensor-core GEMM of the same product (library reference point)
+            try:
+                for _ in range(2):
+                    Ci = torch._int_mm(dA, dB)
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(5):
+                    Ci = torch._int_mm(dA, dB)
+                e1.record()
+                torch.cuda.synchronize()
+                ctx["int8_tensor_core_gemm_TOPS"] = ops / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e12
+                ctx["int8_gemm_equals_awe6"] = bool(torch.equal(Ci, C))
+                parity_ok = parity_ok and ctx["int8_gemm_equals_awe6"]
+                del Ci
+            except Exception as ex:  # library reference point only
+                ctx["int8_tensor_core_gemm_TOPS"] = None
+                ctx["int8_gemm_error"] = str(ex)[:100]
         # the other configurations, device-timed through awe_gemm_exact (context only; their parity is
         # covered by the GPU tests).  Inputs are drawn on the device from a seeded torch generator.
-        if (M, N, K) == (8192, 8192, 8192):
+        if want("configs") and (M, N, K) == (8192, 8192, 8192):
             gen = torch.Generator(device=dev)
             gen.manual_seed(7)
 
@@ -554,7 +592,7 @@ def main():
                                       "residues_GBs": 8192 * 8192 * (8 + nmod) / (ms_res * 1e-3) / 1e9,
                                       "crt_GBs": 8192 * 8192 * (2 * nmod + 16) / (ms_crt * 1e-3) / 1e9}
             del aw, bw, wsw, cw, ra, rc
-        if (M, N, K) == (8192, 8192, 8192):
+        if want("ceiling") and (M, N, K) == (8192, 8192, 8192):
             # FP4 MMA ceiling of this kernel on this part: one raw product on all-zero planes, which
             # draws too little power to be capped, so it shows the structural limit at ~max clock
             kz = 65536
@@ -573,15 +611,17 @@ def main():
             ctx["fp4_ceiling_zero_data_TFLOPs"] = ceil_tflops
             ctx["fp4_ceiling_clock_mhz"] = b.awe_last_gemm_clock_mhz(h)
             line["roofline"]["frac_of_measured_fp4_ceiling"] = gemm_tflops / (ceil_tflops * fmt_scale)
-            del pz
+            del pz, pzo
+        if want("reconstruct") and (M, N, K) == (8192, 8192, 8192):
+            pzo = torch.empty((8192, 8192), dtype=torch.int32, device=dev)
             # stand-alone reconstruction (HBM pass): 6 FP32 product matrices -> int32
             P6 = torch.zeros((6, 8192, 8192), dtype=torch.float32, device=dev)
             for _ in range(2):
-                b.awe_reconstruct(h, enc, 0, P6, 8192 * 8192, 8192, 8192, 8192, pzo, b.C_I32, 8192)
+                b.awe_reconstruct(h, b.ENC_INT8_AWE6, 0, P6, 8192 * 8192, 8192, 8192, 8192, pzo, b.C_I32, 8192)
             torch.cuda.synchronize()
             e0.record()
             for _ in range(5):
-                b.awe_reconstruct(h, enc, 0, P6, 8192 * 8192, 8192, 8192, 8192, pzo, b.C_I32, 8192)
+                b.awe_reconstruct(h, b.ENC_INT8_AWE6, 0, P6, 8192 * 8192, 8192, 8192, 8192, pzo, b.C_I32, 8192)
             e1.record()
             torch.cuda.synchronize()
             ctx["standalone_reconstruct_GBs"] = 8192 * 8192 * 28 / (e0.elapsed_time(e1) / 5 * 1e-3) / 1e9

@@ -31,7 +31,10 @@ __device__ __forceinline__ long long symmetric_mod(long long x, int m) {
 // flight per thread), the sums of the exact encodings with 32-bit output wrap modulo 2^32 exactly
 // like the fused epilogue, and the four results leave as one 16-byte store (two for 64-bit output,
 // one 8-byte store for 16-bit residues).
-__global__ void __launch_bounds__(256)
+// R is the number of products as a compile-time constant (so that no predicated-off slot of a
+// longer unrolled loop is issued), or 0 for any count up to AWE_MAX_PRODUCTS.
+template <int R>
+__global__ void __launch_bounds__(256, R > 0 && R <= 8 ? 3 : 2)
 reconstruct_kernel(const float* __restrict__ P, long long plane_stride, long long ldp, int M, int N,
                    const __grid_constant__ ReconParams p, void* __restrict__ C, long long ldc, int vec_ld, int vec_st) {
     const int groups_per_row = (N + 3) / 4;
@@ -41,15 +44,17 @@ reconstruct_kernel(const float* __restrict__ P, long long plane_stride, long lon
         const int row = (int)(g / groups_per_row), col = (int)(g % groups_per_row) * 4;
         const int n = min(4, N - col);
         const float* src0 = P + (long long)row * ldp + col;
-        float4 v[AWE_MAX_PRODUCTS];
+        constexpr int kSlots = R > 0 ? R : AWE_MAX_PRODUCTS;
+        const int r = R > 0 ? R : p.r;
+        float4 v[kSlots];
         if (vec_ld && n == 4) {
 #pragma unroll
-            for (int k = 0; k < AWE_MAX_PRODUCTS; ++k)
-                if (k < p.r) v[k] = __ldcs(reinterpret_cast<const float4*>(src0 + k * plane_stride));
+            for (int k = 0; k < kSlots; ++k)
+                if (k < r) v[k] = __ldcs(reinterpret_cast<const float4*>(src0 + k * plane_stride));
         } else {
 #pragma unroll
-            for (int k = 0; k < AWE_MAX_PRODUCTS; ++k)
-                if (k < p.r) {
+            for (int k = 0; k < kSlots; ++k)
+                if (k < r) {
                     const float* src = src0 + k * plane_stride;
                     v[k].x = src[0];
                     v[k].y = n > 1 ? src[1] : 0.f;
@@ -62,8 +67,8 @@ reconstruct_kernel(const float* __restrict__ P, long long plane_stride, long lon
             // |D C| < 2^31, so sums taken modulo 2^32 equal D C although single terms may not fit
             uint32_t acc[4] = {0, 0, 0, 0};
 #pragma unroll
-            for (int k = 0; k < AWE_MAX_PRODUCTS; ++k)
-                if (k < p.r) {
+            for (int k = 0; k < kSlots; ++k)
+                if (k < r) {
                     const uint32_t l = (uint32_t)p.ell[k];
                     acc[0] += l * (uint32_t)__float2int_rn(v[k].x);
                     acc[1] += l * (uint32_t)__float2int_rn(v[k].y);
@@ -75,8 +80,8 @@ reconstruct_kernel(const float* __restrict__ P, long long plane_stride, long lon
         } else {
             long long acc[4] = {0, 0, 0, 0};
 #pragma unroll
-            for (int k = 0; k < AWE_MAX_PRODUCTS; ++k)
-                if (k < p.r) {
+            for (int k = 0; k < kSlots; ++k)
+                if (k < r) {
                     const float f[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -136,9 +141,21 @@ extern "C" awe_status_t awe_reconstruct(awe_handle_t h, int enc, int modulus, co
     const size_t elem = out_dt == AWE_C_I64 ? 8 : (out_dt == AWE_C_RES_I16 ? 2 : 4);
     const int vec_st = ((uintptr_t)C_dev % (4 * elem) == 0) && (ldc % 4 == 0);
     const long long total = M * ((N + 3) / 4);
-    const unsigned blocks = (unsigned)std::min<long long>((total + 255) / 256, (long long)h->sm_count * 16);
-    reconstruct_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(P_dev, plane_stride, ldp, (int)M, (int)N, p, C_dev, ldc,
-                                                                 vec_ld, vec_st);
+    const unsigned blocks = (unsigned)std::min<long long>((total + 255) / 256, (long long)h->sm_count * 24);
+    cudaStream_t st = (cudaStream_t)stream;
+#define AWE_RECON(R_) \
+    reconstruct_kernel<R_><<<blocks, 256, 0, st>>>(P_dev, plane_stride, ldp, (int)M, (int)N, p, C_dev, ldc, vec_ld, vec_st)
+    switch (d.r) {
+        case 1: AWE_RECON(1); break;
+        case 3: AWE_RECON(3); break;
+        case 4: AWE_RECON(4); break;
+        case 6: AWE_RECON(6); break;
+        case 8: AWE_RECON(8); break;
+        case 9: AWE_RECON(9); break;
+        case 12: AWE_RECON(12); break;
+        default: AWE_RECON(0); break;
+    }
+#undef AWE_RECON
     if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
     h->launches += 1;
     return AWE_OK;
