@@ -29,8 +29,9 @@
 //
 // Warp roles: warp 0 lane 0 issues TMA loads, warp 1 lane 0 issues MMAs (warp 1 also owns the
 // tensor-memory allocation), warps 2..9 are the epilogue (warp w reads TMEM lanes 32*(w%4)..+31
-// and columns 128*((w-2)/4)..+127).  Every wait is bounded: when one expires the CTA records the
-// site in the status word, raises a shared abort flag and winds down normally.
+// and columns 128*((w-2)/4)..+127).
+// Every wait is bounded: when one expires the CTA records the site in the status word, raises a
+// shared abort flag and winds down normally.
 #include <cuda.h>
 
 #include <algorithm>
@@ -45,6 +46,13 @@ using namespace gemm;
 namespace {
 
 constexpr int kTileN = 256;
+// Accumulator columns per tensor-memory load of the epilogue (16 or 32); also the number of columns
+// the two accumulators share.  16 measured 1.3 % (6-product record) to 2.6 % (residue records) faster
+// than 32: the shared columns are handed back after a smaller load and fewer registers are live.
+#ifndef AWE_DRAIN_COLS
+#define AWE_DRAIN_COLS 16
+#endif
+#define AWE_ACC1_COL (256 - AWE_DRAIN_COLS)
 #ifndef AWE_PAIR_STAGES
 #define AWE_PAIR_STAGES 6
 #endif
@@ -65,12 +73,20 @@ struct Cfg {
         (1u << 4) | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)((kTileM * kCtas) >> 4) << 24);
 };
 constexpr int kMaxStages = 6;
-// Two accumulators of 256 columns and 32 columns of scale bytes do not fit 512 columns side by
-// side, so accumulator 1 starts inside the last 32 columns of accumulator 0.  The epilogue reads
+// Threads per CTA (the variant that forms sum planes adds six warps) and first epilogue warp.
+template <bool kDerive> struct Roles {
+    static constexpr int kThreadsCta = kDerive ? kThreadsDerive : kThreads;
+    static constexpr int kEpiWarp0 = 2;
+};
+// Two accumulators of 256 columns and the columns of scale bytes do not fit 512 columns side by
+// side, so accumulator 1 starts inside the last columns of accumulator 0.  The epilogue reads
 // those shared columns first and releases them separately (overlap_free), which lets the MMAs of
 // the next segment start while the rest of the previous accumulator is still being drained.
+// Constant scale bytes: with a 16-column overlap the second accumulator ends at column 496 and both
+// operands read their (identical) scales from the last 16 columns.
+constexpr uint32_t kSfaMain = AWE_DRAIN_COLS == 32 ? gemm::kSfaCol : 496u, kSfbMain = 496u;
 constexpr uint32_t kAccCol0 = 0;
-constexpr uint32_t kAccCol1 = 224;
+constexpr uint32_t kAccCol1 = AWE_ACC1_COL;
 
 struct Shared {
     uint64_t full[kMaxStages];
@@ -144,21 +160,30 @@ struct EpiMath {
     float acc_scale;
     float mf, inv_m, lo, hi;  // modulus and its symmetric range as floats
     int reduce_each;          // reduce the running residue sum after every segment (very long K only)
+    // Every product of a segment stays below 2^22 in magnitude: adding 1.5 * 2^23 / acc_scale to the
+    // accumulator word leaves the integer product in the low mantissa bits, so the conversion is one
+    // FP32 add and the constant's own bits are taken off the sums once per tile.
+    int use_magic;
+    float magic;
+    uint32_t magic_bits;
 };
 
 // Drain 32 accumulator columns (block BLK of this thread's 128) and fold them into the running sums.
 // When `early_bar` is non-zero these are the columns the two accumulators share: they are handed
 // back to the MMA issuer as soon as they sit in registers, before any arithmetic.
+
+constexpr int kDrainCols = AWE_DRAIN_COLS;  // accumulator columns per tensor-memory load of the epilogue
 template <int BLK>
 __device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128], const EpiMath& em, int ell,
                                             uint32_t early_bar = 0, int lane = 0, bool remote = false) {
-    uint32_t v[32];
-    ptx::tmem_ld_32x32(taddr + BLK * 32, v);
+    uint32_t v[kDrainCols];
+    if (kDrainCols == 32) ptx::tmem_ld_32x32(taddr + BLK * kDrainCols, reinterpret_cast<uint32_t(&)[32]>(v));
+    else ptx::tmem_ld_32x16(taddr + BLK * kDrainCols, reinterpret_cast<uint32_t(&)[16]>(v));
     ptx::tmem_wait_ld();
     if (early_bar) release(early_bar, lane, remote);
     if (em.out_mode == OUT_RAW_F32) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) sum[BLK * 32 + i] = __float_as_uint(__uint_as_float(v[i]) * em.acc_scale);
+        for (int i = 0; i < kDrainCols; ++i) sum[BLK * kDrainCols + i] = __float_as_uint(__uint_as_float(v[i]) * em.acc_scale);
     } else if (em.m) {
         // Running sum kept as a float (exact: |ell| <= m/2, |residue| <= m/2 + 1, few terms).  The
         // accumulator holds P / acc_scale; the scale (a power of two) is folded into the constants:
@@ -168,18 +193,31 @@ __device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128]
         const float q_scale = em.acc_scale * em.inv_m, m_scaled = em.mf / em.acc_scale;
         const float lam = (float)ell * em.acc_scale;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
+        for (int i = 0; i < kDrainCols; ++i) {
             const float a = __uint_as_float(v[i]);
-            const float q = __fadd_rn(__fadd_rn(__fmul_rn(a, q_scale), magic), -magic);
+            const float q = __fadd_rn(__fmaf_rn(a, q_scale, magic), -magic);
             const float res = __fmaf_rn(-q, m_scaled, a);
-            float sf = __fmaf_rn(lam, res, __uint_as_float(sum[BLK * 32 + i]));
+            float sf = __fmaf_rn(lam, res, __uint_as_float(sum[BLK * kDrainCols + i]));
             if (em.reduce_each) sf = mod_symmetric(sf, em.mf, em.inv_m, em.lo, em.hi);
-            sum[BLK * 32 + i] = __float_as_uint(sf);
+            sum[BLK * kDrainCols + i] = __float_as_uint(sf);
         }
+    } else if (em.use_magic) {
+#pragma unroll
+        for (int i = 0; i < kDrainCols; ++i)
+            sum[BLK * kDrainCols + i] += (uint32_t)ell * __float_as_uint(__fadd_rn(__uint_as_float(v[i]), em.magic));
     } else {
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-            sum[BLK * 32 + i] += (uint32_t)ell * (uint32_t)__float2int_rn(__uint_as_float(v[i]) * em.acc_scale);
+        for (int i = 0; i < kDrainCols; ++i)
+            sum[BLK * kDrainCols + i] += (uint32_t)ell * (uint32_t)__float2int_rn(__uint_as_float(v[i]) * em.acc_scale);
+    }
+}
+
+// Blocks FIRST .. LAST-1 of this thread's columns, in order.
+template <int FIRST, int LAST>
+__device__ __forceinline__ void drain_rest(uint32_t taddr, uint32_t (&sum)[128], const EpiMath& em, int ell) {
+    if constexpr (FIRST < LAST) {
+        drain_block<FIRST>(taddr, sum, em, ell);
+        drain_rest<FIRST + 1, LAST>(taddr, sum, em, ell);
     }
 }
 
@@ -189,7 +227,7 @@ __device__ __forceinline__ void drain_block(uint32_t taddr, uint32_t (&sum)[128]
 // kGrouped: the reconstruction is a weighted sum of cells whose own sums fit 32 bits (GemmParams::group_*).
 // kDerive: products with ia2[k] >= 0 multiply sum planes formed in shared memory (pair variant only).
 template <bool kPair, bool kMixed, bool kGrouped, bool kDerive = false>
-__global__ void __launch_bounds__(kDerive ? kThreadsDerive : kThreads, 1)
+__global__ void __launch_bounds__(Roles<kDerive>::kThreadsCta, 1)
 awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a8, const __grid_constant__ CUtensorMap map_b8,
                 const __grid_constant__ GemmParams p) {
@@ -254,10 +292,11 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
     // Constant block scales: every byte of 32 columns x 128 lanes holds the same UE8M0 value,
     // so whatever bytes the MMA picks as scale factors, it reads that value.
-    if (warp >= 2 && warp < 6) {
+    constexpr int kEpiWarp0 = Roles<kDerive>::kEpiWarp0;
+    if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
         const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
-        ptx::tmem_st_fill16(tmem + (lane_base << 16) + kSfaCol, p.sf_word);
-        ptx::tmem_st_fill16(tmem + (lane_base << 16) + kSfbCol, p.sf_word);
+        ptx::tmem_st_fill16(tmem + (lane_base << 16) + kSfaMain, p.sf_word);
+        ptx::tmem_st_fill16(tmem + (lane_base << 16) + kSfbMain, p.sf_word);
         ptx::tmem_wait_st();
     }
     ptx::tc_fence_before();
@@ -365,10 +404,10 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             ptx::mma_f8_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, C::kIdescF8, acc);
                         else if (kPair)
                             ptx::mma_mxf4_pair(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc,
-                                               tmem + kSfaCol, tmem + kSfbCol, acc);
+                                               tmem + kSfaMain, tmem + kSfbMain, acc);
                         else
-                            ptx::mma_mxf4(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc, tmem + kSfaCol,
-                                          tmem + kSfbCol, acc);
+                            ptx::mma_mxf4(tmem + acc_col, a_desc + 2u * j, b_desc + 2u * j, kIdesc, tmem + kSfaMain,
+                                          tmem + kSfbMain, acc);
                     }
                     // frees the stage in both CTAs of a pair
                     if (kPair) ptx::mma_commit_pair(ptx::smem_u32(&sh->empty[s]), 3);
@@ -419,13 +458,13 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 }
             }
         }
-    } else if (kDerive && warp >= 2 + kEpiWarps) {
+    } else if (kDerive && warp >= kEpiWarp0 + kEpiWarps) {
         // -------------------------------------------------------------------- forming warps (kDerive)
         // They follow the producer's sequence of stages.  A stage of a plain product is only passed on;
         // for a product of sum planes the tiles of the following stage are added, 16 bytes at a time,
         // into the stage the MMAs will read (both tiles of a side were written by TMA with the same
         // swizzle, so the sum is elementwise on equal offsets).
-        const int ftid = (int)threadIdx.x - 32 * (2 + kEpiWarps);
+        const int ftid = (int)threadIdx.x - 32 * (kEpiWarp0 + kEpiWarps);
         uint32_t formed_bar[kMaxStages];
         for (int s = 0; s < kStages; ++s) formed_bar[s] = ptx::map_to_cta(ptx::smem_u32(&sh->formed[s]), 0);
         uint32_t it = 0;
@@ -460,9 +499,9 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 }
             }
         }
-    } else {
+    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
         // -------------------------------------------------------------------- epilogue
-        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const int quarter = warp & 3, half = (warp - kEpiWarp0) >> 2;
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)half * 128u;
         const int m = p.modulus;
         // symmetric representative of each coefficient keeps |l_k * residue| below m^2 / 4
@@ -470,7 +509,7 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         uint32_t drains = 0;
         bool ok = true;
         // this warp's 4 KB staging block for the tile write-out
-        uint8_t* stage = smem_raw + (tiles_base - raw) + (size_t)kStages * kStageBytes + (size_t)(warp - 2) * kStageWarpBytes;
+        uint8_t* stage = smem_raw + (tiles_base - raw) + (size_t)kStages * kStageBytes + (size_t)(warp - kEpiWarp0) * kStageWarpBytes;
         // barriers the MMA issuer (CTA 0) waits on
         uint32_t acc_empty_bar[2], overlap_bar = ptx::smem_u32(&sh->overlap_free);
         for (int b = 0; b < 2; ++b) acc_empty_bar[b] = ptx::smem_u32(&sh->acc_empty[b]);
@@ -490,12 +529,16 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // |sum| <= terms * (m/2)^2 must stay below 2^22
             em.reduce_each = (long long)p.r * chunks * (m / 2 + 2) * (m / 2 + 2) >= (1ll << 22);
         }
+        em.use_magic = p.small_sums && !m && !kGrouped && p.out_mode != OUT_RAW_F32;
+        em.magic = 12582912.0f / em.acc_scale;
+        em.magic_bits = __float_as_uint(em.magic);
         for (int t = worker, tile_iter = 0; t < num_tiles && ok; t += num_workers, ++tile_iter) {
             int tm, tn;
             tile_coords(t, p.tiles_m, p.tiles_n, &tm, &tn);
             uint32_t sum[128];
 #pragma unroll
             for (int i = 0; i < 128; ++i) sum[i] = 0;
+            uint32_t magic_corr = 0;  // sum over this tile's drains of l_k * (bit pattern of the conversion constant)
             // ---- tile write-out.  This thread owns one row and 128 consecutive columns; the warp passes
             // every 128-byte row piece through its shared-memory staging block so that each store
             // instruction writes 4 rows x 128 contiguous bytes instead of 32 rows x 16 bytes.
@@ -522,7 +565,11 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 int ell = p.ell[k];
                 if (m && ell > m_hi) ell -= m;
                 const bool f8 = kMixed && p.fp8[k];
-                if (kMixed) em.acc_scale = f8 ? 1.0f : p.acc_scale;
+                if (kMixed) {
+                    em.acc_scale = f8 ? 1.0f : p.acc_scale;
+                    em.magic = 12582912.0f / em.acc_scale;
+                    em.magic_bits = __float_as_uint(em.magic);
+                }
 
                 // the accumulator of a merged set is complete after its last product
                 const bool set_last = kk + 1 == p.r || p.set_id[product_at(kk + 1, tile_iter, p.r)] != p.set_id[k];
@@ -536,18 +583,16 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     // The 32 columns shared by the two accumulators are the last block of accumulator 0
                     // (held by the warps of column half 1) and the first block of accumulator 1 (half 0):
                     // they are read first and handed back at once.
+                    constexpr int kBlocks = 128 / kDrainCols;
                     if (ab == 0) {
-                        drain_block<3>(taddr + kAccCol0, sum, em, ell, half == 1 ? overlap_bar : 0u, lane, kPair);
-                        drain_block<0>(taddr + kAccCol0, sum, em, ell);
-                        drain_block<1>(taddr + kAccCol0, sum, em, ell);
-                        drain_block<2>(taddr + kAccCol0, sum, em, ell);
+                        drain_block<kBlocks - 1>(taddr + kAccCol0, sum, em, ell, half == 1 ? overlap_bar : 0u, lane, kPair);
+                        drain_rest<0, kBlocks - 1>(taddr + kAccCol0, sum, em, ell);
                     } else {
                         drain_block<0>(taddr + kAccCol1, sum, em, ell, half == 0 ? overlap_bar : 0u, lane, kPair);
-                        drain_block<1>(taddr + kAccCol1, sum, em, ell);
-                        drain_block<2>(taddr + kAccCol1, sum, em, ell);
-                        drain_block<3>(taddr + kAccCol1, sum, em, ell);
+                        drain_rest<1, kBlocks>(taddr + kAccCol1, sum, em, ell);
                     }
                     release(acc_empty_bar[ab], lane, kPair);
+                    if (em.use_magic) magic_corr += (uint32_t)ell * em.magic_bits;
                 }
                 if (kGrouped) {
                     // A group of the grouped reconstruction is complete when the next product belongs to
@@ -565,6 +610,10 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
             if (!ok) break;
             if (kGrouped) continue;  // everything has been written group by group
+            if (em.use_magic) {
+#pragma unroll
+                for (int i = 0; i < 128; ++i) sum[i] -= magic_corr;
+            }
             if (m) {
                 // residue sums are floats: one last reduction, then to integers in the symmetric range
 #pragma unroll
@@ -655,7 +704,7 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
     const int workers = std::min(p.tiles_m * p.tiles_n, h->sm_count / C::kCtas);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(workers * C::kCtas));
-    cfg.blockDim = dim3(kDerive ? kThreadsDerive : kThreads);
+    cfg.blockDim = dim3(Roles<kDerive>::kThreadsCta);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -880,6 +929,17 @@ awe_status_t awe::gemm_planes_window(awe_ctx* h, int enc, int modulus, PlaneWind
         p.kblock0 = (int)kb0;
         p.num_kblocks = (int)std::min(seg_kblocks, total_kblocks - kb0);
         p.accumulate = kb0 > 0;
+        {
+            // largest |accumulator| at a drain: products of one set (n_g of them) over one segment
+            int n_g = 1;
+            for (int k = 0; k < d.r; ++k) {
+                int run = 0;
+                for (int j = 0; j < d.r; ++j) run += p.set_id[j] == p.set_id[k];
+                n_g = std::max(n_g, run);
+            }
+            const int64_t seg_len = 256 * (int64_t)std::min(p.num_kblocks, p.chunk_kblocks);
+            p.small_sums = (int64_t)n_g * d.c_a * d.c_b * seg_len < ((int64_t)1 << 22);
+        }
         if (mixed) {
             // an E4M3 K block holds 128 elements, an E2M1 block 256
             p.kblock0_8 = 2 * p.kblock0;

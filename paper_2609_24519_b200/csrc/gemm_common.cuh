@@ -56,6 +56,9 @@ struct GemmParams {
     // Sum planes formed in the kernel: product k multiplies (plane ia[k] + plane ia2[k]) of A by
     // (plane ib[k] + plane ib2[k]) of B when ia2[k] >= 0 (then ib2[k] >= 0 too); -1 otherwise.
     int ia2[AWE_MAX_PRODUCTS], ib2[AWE_MAX_PRODUCTS];
+    // every accumulator of this launch stays below 2^22 in magnitude when it is drained (Section 3.4's bound
+    // with the segment length of this launch): lets the epilogue convert with one FP32 add
+    int small_sums;
 };
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
