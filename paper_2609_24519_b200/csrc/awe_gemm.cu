@@ -244,7 +244,10 @@ __device__ __forceinline__ void drain_rest(uint32_t taddr, uint32_t (&sum)[128],
 // itself); the others are E2M1 products as above.  Pair variant only.
 // kGrouped: the reconstruction is a weighted sum of cells whose own sums fit 32 bits (GemmParams::group_*).
 // kDerive: products with ia2[k] >= 0 multiply sum planes formed in shared memory (pair variant only).
-template <bool kPair, bool kMixed, bool kGrouped, bool kDerive = false, int kEpi = kEpiAny>
+// kOut: the output element type the tile write-out is compiled for (kOutAny: chosen at run time).
+// With all three write-outs in one kernel the compiler spills ten times as much of the running sums.
+enum OutSel { kOutAny = -1, kOut32 = 0, kOut64 = 1, kOut16 = 2 };
+template <bool kPair, bool kMixed, bool kGrouped, bool kDerive = false, int kEpi = kEpiAny, int kOut = kOutAny>
 __global__ void __launch_bounds__(Roles<kDerive>::kThreadsCta, 1)
 awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a8, const __grid_constant__ CUtensorMap map_b8,
@@ -647,7 +650,8 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     sum[i] = __float_as_uint(mod_symmetric(__uint_as_float(sum[i]), em.mf, em.inv_m, em.lo, em.hi) +
                                              12582912.0f) - 0x4B400000u;  // float -> int
             }
-            if (p.out_mode == OUT_I32 || p.out_mode == OUT_RES_I32 || p.out_mode == OUT_RAW_F32) {
+            if ((kOut == kOutAny || kOut == kOut32) &&
+                (p.out_mode == OUT_I32 || p.out_mode == OUT_RES_I32 || p.out_mode == OUT_RAW_F32)) {
                 uint8_t* gbase = reinterpret_cast<uint8_t*>(p.C) + (row0 * p.ldc + col0) * 4;
 #pragma unroll
                 for (int blk = 0; blk < 4; ++blk) {  // 32 columns = 128 bytes per row
@@ -664,9 +668,9 @@ awe_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     store_rows_128b<4>(stage, lane, chunk, gbase + blk * 128, p.ldc * 4, rows_valid,
                                        (p.N - col0 - blk * 32) * 4, p.vec_store, false);
                 }
-            } else if (p.out_mode == OUT_I64) {
+            } else if ((kOut == kOutAny || kOut == kOut64) && p.out_mode == OUT_I64) {
                 write_i64(1, p.accumulate != 0);
-            } else {  // OUT_RES_I16
+            } else if (kOut == kOutAny || kOut == kOut16) {  // OUT_RES_I16
                 uint8_t* gbase = reinterpret_cast<uint8_t*>(p.C) + (row0 * p.ldc + col0) * 2;
 #pragma unroll
                 for (int blk = 0; blk < 2; ++blk) {  // 64 columns = 128 bytes per row
@@ -712,13 +716,13 @@ bool use_pairs() {
     return v;
 }
 
-template <bool kPair, bool kMixed, bool kGrouped = false, bool kDerive = false, int kEpi = kEpiAny>
+template <bool kPair, bool kMixed, bool kGrouped = false, bool kDerive = false, int kEpi = kEpiAny, int kOut = kOutAny>
 awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ma8,
                             const CUtensorMap& mb8, GemmParams& p, cudaStream_t st) {
     using C = Cfg<kPair>;
-    bool& attr_set = h->smem_attr_set[(kEpi == kEpiResidue ? 6 : (kDerive ? 5 : (kGrouped ? 4 : (kMixed ? 3 : (kPair ? 0 : 1)))))];
+    bool& attr_set = h->smem_attr_set[(kOut + 1) * 8 + (kEpi == kEpiResidue ? 6 : (kDerive ? 5 : (kGrouped ? 4 : (kMixed ? 3 : (kPair ? 0 : 1)))))];
     if (!attr_set) {
-        if (cudaFuncSetAttribute(awe_gemm_kernel<kPair, kMixed, kGrouped, kDerive, kEpi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(awe_gemm_kernel<kPair, kMixed, kGrouped, kDerive, kEpi, kOut>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)C::kSmemBytes) != cudaSuccess)
             return AWE_ERR_CUDA;
         attr_set = true;
@@ -740,7 +744,7 @@ awe_status_t launch_variant(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair, kMixed, kGrouped, kDerive, kEpi>, ma, mb, ma8, mb8, p);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, awe_gemm_kernel<kPair, kMixed, kGrouped, kDerive, kEpi, kOut>, ma, mb, ma8, mb8, p);
     if (err != cudaSuccess) {
         if (getenv("AWE_DEBUG")) fprintf(stderr, "awe: GEMM launch failed: %s\n", cudaGetErrorString(err));
         return AWE_ERR_CUDA;
@@ -755,19 +759,27 @@ awe_status_t launch_gemm(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& m
     for (int k = 0; k < p.r; ++k) derive = derive || p.ia2[k] >= 0;
     if (derive) return launch_variant<true, false, false, true>(h, ma, mb, ma, mb, p, st);
     if (!use_pairs()) return launch_variant<false, false>(h, ma, mb, ma, mb, p, st);
-    // residue records get an epilogue specialised at compile time
+    // the plain pair kernel is compiled per output type, residue records also with their own arithmetic
     if (p.modulus && (p.out_mode == OUT_RES_I16 || p.out_mode == OUT_RES_I32)) {
         const long long chunks = (p.num_kblocks + p.chunk_kblocks - 1) / p.chunk_kblocks, half_m = p.modulus / 2 + 2;
-        if ((long long)p.r * chunks * half_m * half_m < (1ll << 22))  // no reduction needed between segments
-            return launch_variant<true, false, false, false, kEpiResidue>(h, ma, mb, ma, mb, p, st);
+        if ((long long)p.r * chunks * half_m * half_m < (1ll << 22)) {  // no reduction needed between segments
+            return p.out_mode == OUT_RES_I16
+                       ? launch_variant<true, false, false, false, kEpiResidue, kOut16>(h, ma, mb, ma, mb, p, st)
+                       : launch_variant<true, false, false, false, kEpiResidue, kOut32>(h, ma, mb, ma, mb, p, st);
+        }
     }
-    return launch_variant<true, false>(h, ma, mb, ma, mb, p, st);
+    switch (p.out_mode) {
+        case OUT_I64: return launch_variant<true, false, false, false, kEpiAny, kOut64>(h, ma, mb, ma, mb, p, st);
+        case OUT_RES_I16: return launch_variant<true, false, false, false, kEpiAny, kOut16>(h, ma, mb, ma, mb, p, st);
+        default: return launch_variant<true, false, false, false, kEpiAny, kOut32>(h, ma, mb, ma, mb, p, st);
+    }
 }
 
 // Records with E4M3 products: (ma, mb) cover the E2M1 planes, (ma8, mb8) the E4M3 planes.
 awe_status_t launch_gemm_mixed(awe_ctx* h, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ma8,
                                const CUtensorMap& mb8, GemmParams& p, cudaStream_t st) {
-    return launch_variant<true, true>(h, ma, mb, ma8, mb8, p, st);
+    if (p.out_mode == OUT_I64) return launch_variant<true, true, false, false, kEpiAny, kOut64>(h, ma, mb, ma8, mb8, p, st);
+    return launch_variant<true, true, false, false, kEpiAny, kOut32>(h, ma, mb, ma8, mb8, p, st);
 }
 
 int b_box_rows() { return use_pairs() ? Cfg<true>::kBRows : Cfg<false>::kBRows; }

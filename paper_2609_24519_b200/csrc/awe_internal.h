@@ -102,7 +102,7 @@ struct awe_ctx {
     cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_done = nullptr;
     cudaEvent_t ev_a[kMaxHostChunks] = {nullptr}, ev_bcol[kMaxHostColBlocks] = {nullptr};
     cudaEvent_t ev_c[kMaxHostChunks * kMaxHostColBlocks] = {nullptr};
-    bool smem_attr_set[8] = {false, false, false, false, false, false, false, false};  // dynamic shared-memory limit raised (per kernel, this device)
+    bool smem_attr_set[32] = {false};  // dynamic shared-memory limit raised (per kernel, this device)
 };
 
 namespace awe {
