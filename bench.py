@@ -369,23 +369,6 @@ def main():
                             "peak": peaks["hbm_gbs"], "unit": "GB/s"},
     }
     line["encode_roofline"]["frac"] = line["encode_roofline"]["achieved"] / peaks["hbm_gbs"]
-    # The encode writes 3 bytes for every byte it reads, and HBM writes alone run well below the
-    # read+write copy figure: measure a plain fill of the same size and report the write stream against it.
-    fill_buf = torch.empty(plane_bytes, dtype=torch.uint8, device=dev)
-    for _ in range(3):
-        fill_buf.fill_(1)
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    f0.record()
-    for _ in range(10):
-        fill_buf.fill_(1)
-    f1.record()
-    torch.cuda.synchronize()
-    fill_gbs = fill_buf.numel() / (f0.elapsed_time(f1) / 10 * 1e-3) / 1e9
-    enc_write_gbs = fill_buf.numel() / (ms_encode * 1e-3) / 1e9
-    line["encode_roofline"].update({"write_GBs": enc_write_gbs, "fill_GBs_measured_now": fill_gbs,
-                                    "frac_of_write_bandwidth": enc_write_gbs / fill_gbs})
-    del fill_buf
 
     def want(name):
         return args.context == "all" or name in args.context.split(",")

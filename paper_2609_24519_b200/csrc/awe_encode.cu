@@ -20,9 +20,6 @@ namespace {
 
 constexpr int kEncThreads = 256;
 constexpr size_t kLutSmemBytes = 256 * 128;
-#ifndef AWE_ENC_BLOCKS_PER_SM
-#define AWE_ENC_BLOCKS_PER_SM 7
-#endif
 #ifndef AWE_KXR_LANES_K
 #define AWE_KXR_LANES_K 4
 #endif
@@ -37,10 +34,14 @@ __device__ __forceinline__ void load_lut(unsigned char* lut_s, const uint64_t* _
         for (int i = threadIdx.x; i < 256 * 16; i += blockDim.x) d[i] = lut_g[i >> 4];
     } else {
         uint32_t* d = reinterpret_cast<uint32_t*>(lut_s);
-        for (int i = threadIdx.x; i < 256 * 32; i += blockDim.x) {
-            const uint64_t e = lut_g[i >> 5];
+        // a warp reads 32 entries with one load and hands each to all lanes in turn
+        const int lane = threadIdx.x & 31;
+        for (int e0 = (threadIdx.x >> 5) * 32; e0 < 256; e0 += (blockDim.x >> 5) * 32) {
+            const uint64_t e = lut_g[e0 + lane];
             // planes 0-3 stay in the low nibbles of bytes 0-3; planes 4, 5 move to the high nibbles of bytes 0, 1
-            d[i] = (uint32_t)e | (((uint32_t)(e >> 32) & 0x0F0Fu) << 4);
+            const uint32_t c = (uint32_t)e | (((uint32_t)(e >> 32) & 0x0F0Fu) << 4);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) d[(e0 + i) * 32 + lane] = __shfl_sync(0xFFFFFFFFu, c, i);
         }
     }
     __syncthreads();
@@ -448,16 +449,32 @@ encode16_kxr_kernel(const uint16_t* __restrict__ X, int64_t R, int64_t K, int64_
     }
 }
 
+// Grid: kBlocksPerSm blocks per SM is what the tables allow (7 x 32 KB of shared memory).  Registers
+// let fewer be resident at once (5 of the 6-plane RxK kernel, 3 of the transposing one) and the rest
+// follow as a second wave; measured at 8192 x 8192 that is still faster for 5 planes and more and for
+// every transposing kernel (60 against 76 us for 6 planes) than a grid of resident blocks only, while
+// the RxK kernels of up to 4 planes gain 2-3 us from a grid of exactly the resident blocks.
+constexpr int kBlocksPerSm = 7;
+
+template <typename Kernel>
+int resident_blocks(Kernel kernel, size_t smem) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kEncThreads, smem) != cudaSuccess || n < 1)
+        n = kBlocksPerSm;
+    return std::min(n, kBlocksPerSm);
+}
+
 template <int NP>
 cudaError_t launch16(awe_layout_t layout, const uint16_t* X, int64_t R, int64_t K, int64_t ld, const uint64_t* lut,
                      uint8_t* planes, int64_t pitch, int64_t plane_stride, int vec_ok, int sm_count,
                      cudaStream_t stream) {
     const int64_t warps_per_block = kEncThreads / 32;
+    constexpr int kRows = (32 / kKxrLanesK) * 2;
     const int64_t items = layout == AWE_ROWMAJOR_RxK
                               ? R * ((pitch * 2 + 1023) / 1024)
-                              : ((pitch * 2 + kKxrK - 1) / kKxrK) * ((R + (32 / kKxrLanesK) * 2 - 1) / ((32 / kKxrLanesK) * 2));
+                              : ((pitch * 2 + kKxrK - 1) / kKxrK) * ((R + kRows - 1) / kRows);
     const int64_t blocks =
-        std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
+        std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * kBlocksPerSm);
     if (layout == AWE_ROWMAJOR_RxK)
         encode16_rxk_kernel<NP><<<(unsigned)blocks, kEncThreads, kLut16SmemBytes, stream>>>(X, R, K, ld, lut, planes, pitch,
                                                                                            plane_stride, vec_ok);
@@ -473,13 +490,17 @@ cudaError_t launch(awe_layout_t layout, const int8_t* X, int64_t R, int64_t K, i
                    cudaStream_t stream) {
     const int64_t warps_per_block = kEncThreads / 32;
     if (layout == AWE_ROWMAJOR_RxK) {
+        static const int per_sm = (NP <= 4 && !kMixed)
+                                      ? resident_blocks(encode_rxk_kernel<NP, kMixed, kPacked>, kLutSmemBytes)
+                                      : kBlocksPerSm;
         const int64_t items = R * ((pitch * 2 + 1023) / 1024);
-        const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
+        const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * per_sm);
         encode_rxk_kernel<NP, kMixed, kPacked><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
             X, R, K, ld, lut, planes, planes4, pitch, plane_stride, vec_ok);
     } else {
         const int64_t items = ((pitch * 2 + kKxrK - 1) / kKxrK) * ((R + kKxrRows - 1) / kKxrRows);
-        const int64_t blocks = std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * AWE_ENC_BLOCKS_PER_SM);
+        const int64_t blocks =
+            std::min<int64_t>((items + warps_per_block - 1) / warps_per_block, (int64_t)sm_count * kBlocksPerSm);
         encode_kxr_kernel<NP, kMixed, kPacked><<<(unsigned)blocks, kEncThreads, kLutSmemBytes, stream>>>(
             X, R, K, ld, lut, planes, planes4, pitch, plane_stride, vec_ok);
     }
