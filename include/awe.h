@@ -249,8 +249,9 @@ size_t awe_wide_workspace_bytes(int64_t M, int64_t N, int64_t K);
  * the residue arrays keep the layout of X.  X_dev 16-B aligned, res_dev 4-B aligned. */
 awe_status_t awe_wide_residues(awe_handle_t h, const int64_t* X_dev, int64_t count, int8_t* res_dev, void* stream);
 
-/* Chinese-remainder reconstruction: res_dev[t * count + i] (int16) is the symmetric residue of the
- * unknown integer x_i modulo m_t; writes x_i, the representative with |x_i| <= prod(m)/2, as a
+/* Chinese-remainder reconstruction: res_dev[t * count + i] (int16) is a residue of the unknown integer
+ * x_i modulo m_t (the products deliver the symmetric one; any representative that fits 16 bits is
+ * accepted); writes x_i, the representative with |x_i| <= prod(m)/2, as a
  * 128-bit two's-complement integer: out_dev[2 i] = low 64 bits, out_dev[2 i + 1] = high 64 bits. */
 awe_status_t awe_wide_crt(awe_handle_t h, const int16_t* res_dev, int64_t count, int64_t* out_dev, void* stream);
 

@@ -13,201 +13,223 @@ namespace {
 
 constexpr int kMaxModuli = 32;
 // 5 one-product, 13 three-product and 4 four-product moduli; product = 2^122.86.
-const int kWideModuli[] = {7, 8, 9, 11, 13, 41, 43, 47, 53, 59, 61, 67, 71, 73, 79, 83, 85, 89, 139, 149, 151, 157};
-constexpr int kNumWideModuli = sizeof(kWideModuli) / sizeof(int);
+constexpr int kNumWideModuli = 22;
+constexpr int kWideModuli[kNumWideModuli] = {7,  8,  9,  11, 13, 41, 43, 47, 53,  59,  61,
+                                             67, 71, 73, 79, 83, 85, 89, 139, 149, 151, 157};
 
 typedef unsigned __int128 u128;
 typedef __int128 i128;
 
+// 2^e mod m in the symmetric range, as a float.
+constexpr float pow2_mod_symmetric(int e, int m) {
+    int r = 1 % m;
+    for (int i = 0; i < e; ++i) r = (2 * r) % m;
+    return (float)(r > m / 2 ? r - m : r);
+}
+
+// Built-in modulus number T with the constants of its residue computation, all compile-time.
+template <int T>
+struct WideModulus {
+    static constexpr int m = kWideModuli[T];
+    static constexpr float mf = (float)m, inv_m = 1.0f / (float)m;
+    static constexpr float c1 = pow2_mod_symmetric(14, m), c2 = pow2_mod_symmetric(28, m),
+                           c3 = pow2_mod_symmetric(42, m);
+};
+
 struct ResidueParams {
-    int n;
-    // per modulus, as floats: m, 1/m, 2^14, 2^28, 2^42 mod m, and the symmetric range
-    float mf[kMaxModuli], inv_m[kMaxModuli], c1f[kMaxModuli], c2f[kMaxModuli], c3f[kMaxModuli];
-    float lo[kMaxModuli], hi[kMaxModuli];
+    unsigned int mask;                // bit T: built-in modulus T is wanted
+    long long offset[kNumWideModuli]; // its residues start at out + offset[T]
 };
 
-// |x| < 2^56 as four 14-bit limbs l0..l3: |x| = l0 + l1 2^14 + l2 2^28 + l3 2^42.
-struct Limbs14 {
-    unsigned int l0, l1, l2, l3;
-    bool neg;
-};
+constexpr float kRoundMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds |v| < 2^22 to an integer held in the low mantissa bits
 
-__device__ __forceinline__ Limbs14 split14(long long x) {
+// x mod m for built-in modulus T, on the FP32 pipe.  f holds the four signed 14-bit limbs of x as floats
+// (x = f0 + f1 2^14 + f2 2^28 + f3 2^42).  s = f0 + f1 c1 + f2 c2 + f3 c3 with c_k = 2^(14k) mod m taken
+// in the symmetric range is an integer of magnitude below 2^14 (1 + 3 m / 2) < 2^22, hence exact;
+// q = round(s / m) by one FMA with the rounding constant (the estimate s * (1/m) is off by less than
+// 0.23 / m while every non-integer multiple of 1/m is at least 0.5 / m away from a rounding boundary, so
+// q is the exact nearest integer, either neighbour on a tie); r = s - q m is then exact with
+// |r| <= m / 2, which is the symmetric range except for r = +m/2 of an even modulus.  Returns
+// r + 1.5 * 2^23 as bits: the low byte is r in two's complement.
+template <int T>
+__device__ __forceinline__ uint32_t symmetric_residue_bits(const float (&f)[4]) {
+    typedef WideModulus<T> W;
+    const float s = __fmaf_rn(f[3], W::c3, __fmaf_rn(f[2], W::c2, __fmaf_rn(f[1], W::c1, f[0])));
+    const float q = __fadd_rn(__fmaf_rn(s, W::inv_m, kRoundMagic), -kRoundMagic);
+    float r = __fmaf_rn(-q, W::mf, s);
+    if (W::m % 2 == 0) r = (r == (float)(W::m / 2)) ? -r : r;
+    return __float_as_uint(__fadd_rn(r, kRoundMagic));
+}
+
+// Signed 14-bit limbs of x (|x| < 2^56) as floats: a limb l < 2^14 placed in the mantissa of 2^23 reads
+// as 2^23 + l, and one FMA with +-1 removes the offset and applies the sign of x.
+__device__ __forceinline__ void split14_signed(long long x, float (&f)[4]) {
     const unsigned long long ax = x < 0 ? (unsigned long long)(-x) : (unsigned long long)x;
-    Limbs14 r;
-    r.l0 = (unsigned int)ax & 0x3FFFu;
-    r.l1 = (unsigned int)(ax >> 14) & 0x3FFFu;
-    r.l2 = (unsigned int)(ax >> 28) & 0x3FFFu;
-    r.l3 = (unsigned int)(ax >> 42) & 0x3FFFu;
-    r.neg = x < 0;
-    return r;
+    const float sgn = x < 0 ? -1.0f : 1.0f, off = x < 0 ? 8388608.0f : -8388608.0f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t limb = (uint32_t)(ax >> (14 * k)) & 0x3FFFu;
+        f[k] = __fmaf_rn(__uint_as_float(0x4B000000u | limb), sgn, off);
+    }
 }
 
-// x mod m in the symmetric range, on the FP32 pipe (twice the issue rate of 32-bit integer
-// multiplies).  f holds the signed limbs as floats; s = f0 + f1 c1 + f2 c2 + f3 c3 is an integer below 2^24 in magnitude, hence
-// exact; q = round(s / m) by adding and subtracting 1.5 * 2^23, r = s - q m by one exact FMA, and one
-// correction each way puts r into [-floor(m/2), ceil(m/2) - 1] even if q was off by one.  Returns r
-// as the low byte of (r + 1.5 * 2^23)'s bit pattern, i.e. r in two's complement.
-__device__ __forceinline__ uint32_t symmetric_residue_f(const float (&f)[4], float m, float inv_m, float c1, float c2,
-                                                        float c3, float lo, float hi) {
-    const float magic = 12582912.0f;
-    const float sres = __fmaf_rn(f[3], c3, __fmaf_rn(f[2], c2, __fmaf_rn(f[1], c1, f[0])));
-    const float q = __fadd_rn(__fadd_rn(__fmul_rn(sres, inv_m), magic), -magic);
-    float r = __fmaf_rn(-q, m, sres);
-    r = r > hi ? r - m : r;
-    r = r < lo ? r + m : r;
-    return __float_as_uint(r + magic) & 0xFFu;
+constexpr int kResPerThread = 8;  // consecutive elements per thread: one 8-byte store per modulus
+
+template <int T>
+__device__ __forceinline__ void residues_of_group(const float (&f)[kResPerThread][4], const ResidueParams& p,
+                                                  int8_t* out, long long i0, long long count, bool full) {
+    if (p.mask >> T & 1u) {  // the same for every thread
+        uint32_t word[kResPerThread / 4];
+#pragma unroll
+        for (int w = 0; w < kResPerThread / 4; ++w) {
+            const uint32_t b0 = symmetric_residue_bits<T>(f[4 * w]), b1 = symmetric_residue_bits<T>(f[4 * w + 1]);
+            const uint32_t b2 = symmetric_residue_bits<T>(f[4 * w + 2]), b3 = symmetric_residue_bits<T>(f[4 * w + 3]);
+            word[w] = __byte_perm(__byte_perm(b0, b1, 0x0040), __byte_perm(b2, b3, 0x0040), 0x5410);
+        }
+        int8_t* dst = out + p.offset[T] + i0;
+        if (full) {
+            *reinterpret_cast<uint2*>(dst) = make_uint2(word[0], word[1]);
+        } else {
+            for (int j = 0; j < kResPerThread; ++j)
+                if (i0 + j < count) dst[j] = (int8_t)(word[j / 4] >> (8 * (j % 4)));
+        }
+    }
+    if constexpr (T + 1 < kNumWideModuli) residues_of_group<T + 1>(f, p, out, i0, count, full);
 }
 
-// X: `count` 64-bit integers; out[t * count + i] = symmetric residue of X[i] modulo m[t].
-// A thread takes 4 consecutive elements so every store is a 4-byte word and a warp writes 128
-// contiguous bytes per modulus.
+// X: `count` 64-bit integers; out[offset[T] + i] = symmetric residue of X[i] modulo built-in modulus T
+// for every T in the mask.  A thread takes 8 consecutive elements so every store is an 8-byte word and a
+// warp writes 256 contiguous bytes per modulus; the loop over the moduli is unrolled at compile time, so
+// their constants are immediates.  `vec`: every modulus' array starts on an 8-byte boundary.
 __global__ void __launch_bounds__(256)
 wide_residues_kernel(const long long* __restrict__ X, long long count, const __grid_constant__ ResidueParams p,
-                     int8_t* __restrict__ out) {
-    const long long groups = (count + 3) / 4;
+                     int8_t* __restrict__ out, int vec) {
+    const long long groups = (count + kResPerThread - 1) / kResPerThread;
     for (long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
          g += (long long)gridDim.x * blockDim.x) {
-        const long long i0 = g * 4;
-        long long x[4] = {0, 0, 0, 0};
-        if (i0 + 4 <= count) {
-            const longlong2 a = __ldg(reinterpret_cast<const longlong2*>(X + i0));
-            const longlong2 b = __ldg(reinterpret_cast<const longlong2*>(X + i0) + 1);
-            x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
-        } else {
-            for (int j = 0; j < 4; ++j)
-                if (i0 + j < count) x[j] = X[i0 + j];
-        }
-        float f[4][4];  // signed 14-bit limbs of the four elements
+        const long long i0 = g * kResPerThread;
+        long long x[kResPerThread];
+        if (i0 + kResPerThread <= count) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const Limbs14 v = split14(x[j]);
-            const float sgn = v.neg ? -1.0f : 1.0f;
-            f[j][0] = sgn * (float)v.l0;
-            f[j][1] = sgn * (float)v.l1;
-            f[j][2] = sgn * (float)v.l2;
-            f[j][3] = sgn * (float)v.l3;
-        }
-        const bool full = (i0 + 4 <= count) && ((count & 3) == 0);
-#pragma unroll 2
-        for (int t = 0; t < p.n; ++t) {
-            const float m = p.mf[t], inv_m = p.inv_m[t], c1 = p.c1f[t], c2 = p.c2f[t], c3 = p.c3f[t];
-            const float lo = p.lo[t], hi = p.hi[t];
-            uint32_t word = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) word |= symmetric_residue_f(f[j], m, inv_m, c1, c2, c3, lo, hi) << (8 * j);
-            int8_t* dst = out + (long long)t * count + i0;
-            if (full) {
-                *reinterpret_cast<uint32_t*>(dst) = word;
-            } else {
-                for (int j = 0; j < 4; ++j)
-                    if (i0 + j < count) dst[j] = (int8_t)(word >> (8 * j));
+            for (int j = 0; j < kResPerThread / 2; ++j) {
+                const longlong2 a = __ldg(reinterpret_cast<const longlong2*>(X + i0) + j);
+                x[2 * j] = a.x;
+                x[2 * j + 1] = a.y;
             }
+        } else {
+            for (int j = 0; j < kResPerThread; ++j) x[j] = i0 + j < count ? X[i0 + j] : 0;
         }
+        float f[kResPerThread][4];  // signed 14-bit limbs of the elements
+#pragma unroll
+        for (int j = 0; j < kResPerThread; ++j) split14_signed(x[j], f[j]);
+        residues_of_group<0>(f, p, out, i0, count, vec && i0 + kResPerThread <= count);
     }
 }
 
 struct CrtParams {
-    int n;
-    int m[kMaxModuli];
-    unsigned int w[kMaxModuli][4];  // W_t = (M/m_t) ((M/m_t)^-1 mod m_t) < 2^123 in four 32-bit limbs
-    unsigned int M[4];              // M = prod m_t
+    unsigned int mask;                  // bit T: built-in modulus T takes part
+    long long offset[kNumWideModuli];   // its residues start at res + offset[T] (elements)
+    int w[kNumWideModuli][4];           // W_T = (M/m_T) ((M/m_T)^-1 mod m_T) < 2^123 in four 31-bit limbs
+    int M[4];                           // M = prod m_T in 31-bit limbs
     unsigned long long M_lo, M_hi, half_lo, half_hi;
-    double M_as_double;
+    double inv_M;                       // 1 / M rounded to double
 };
 
-// res[t * count + i]: symmetric residues of the unknown integers modulo m_t.  The integer with
-// -M/2 < x <= M/2 is x = sum_t r_t W_t mod M (textbook CRT) with r_t taken in [0, m_t).  The sum is
-// formed limb by limb (four 64-bit accumulators of 32 x 32-bit products, no carries needed: 22 terms
-// below 2^40 each), the quotient by M (< 2^13) is estimated in double precision, q M is subtracted
-// limb by limb, carries are propagated once, and at most two corrections fix the estimate.
-constexpr int kCrtBatch = 12;
-
-// One element: x in (-M/2, M/2] from the four limb sums a0..a3 of sum_t r_t W_t.
-__device__ __forceinline__ i128 crt_reduce(unsigned long long a0, unsigned long long a1, unsigned long long a2,
-                                           unsigned long long a3, const CrtParams& p, i128 M, i128 half) {
-    const double xd = ((double)a3 * 4294967296.0 + (double)a2) * 18446744073709551616.0 +
-                      (double)a1 * 4294967296.0 + (double)a0;
-    const long long q = (long long)floor(xd / p.M_as_double);
-    // d_k = a_k - q M_k (|d_k| < 2^46), then x - q M = sum_k d_k 2^(32 k) with signed carries
-    long long c = (long long)a0 - q * (long long)p.M[0];
-    const unsigned long long r0 = (unsigned long long)c & 0xFFFFFFFFull;
-    c = (c >> 32) + (long long)a1 - q * (long long)p.M[1];
-    const unsigned long long r1 = (unsigned long long)c & 0xFFFFFFFFull;
-    c = (c >> 32) + (long long)a2 - q * (long long)p.M[2];
-    const unsigned long long r2 = (unsigned long long)c & 0xFFFFFFFFull;
-    c = (c >> 32) + (long long)a3 - q * (long long)p.M[3];  // top limb: signed, |c| < 2^28, so its low 32 bits
-    // placed at bit 96 give the right two's-complement value even when the estimate was one too large
-    i128 x = (i128)(((u128)(unsigned long long)c << 96) | ((u128)r2 << 64) | ((u128)r1 << 32) | (u128)r0);
+// res[offset[T] + i]: residues of the unknown integers modulo m_T (any representative that fits 16 bits;
+// the products deliver the symmetric one).  The integer with -M/2 < x <= M/2 is x = sum_T r_T W_T mod M
+// (textbook CRT).  The sum is formed limb by limb with signed 32 x 32 -> 64-bit multiply-adds (W_T in
+// 31-bit limbs so that they are positive as signed words; 22 terms below 2^46 each, no carries needed),
+// the quotient by M (|q| < 2^20) is estimated in double precision (one multiplication by 1/M: off by at
+// most one), q M is subtracted limb by limb, carries are propagated once, and at most two corrections
+// fix the estimate.  (The same sums as exact FP32 FMAs over 12-bit limbs of W_T, 11 per residue instead
+// of 4 multiply-adds, were measured slower: 1.43 against 1.16 ms for 8192 x 8192 results.)
+__device__ __forceinline__ i128 crt_reduce(const long long (&a)[4], const CrtParams& p, i128 M, i128 half) {
+    const double two31 = 2147483648.0;
+    const double xd = (((double)a[3] * two31 + (double)a[2]) * two31 + (double)a[1]) * two31 + (double)a[0];
+    const long long q = (long long)floor(xd * p.inv_M);
+    // d_k = a_k - q M_k (|d_k| < 2^52), then x - q M = sum_k d_k 2^(31 k) with signed carries
+    long long c = a[0] - q * (long long)p.M[0];
+    const unsigned long long r0 = (unsigned long long)c & 0x7FFFFFFFull;
+    c = (c >> 31) + a[1] - q * (long long)p.M[1];
+    const unsigned long long r1 = (unsigned long long)c & 0x7FFFFFFFull;
+    c = (c >> 31) + a[2] - q * (long long)p.M[2];
+    const unsigned long long r2 = (unsigned long long)c & 0x7FFFFFFFull;
+    c = (c >> 31) + a[3] - q * (long long)p.M[3];  // top limb: signed and small, since |x - q M| < 2 M < 2^124
+    i128 x = (i128)c * ((i128)1 << 93) + (i128)(((u128)r2 << 62) | ((u128)r1 << 31) | (u128)r0);
     if (x < 0) x += M;
     if (x >= M) x -= M;
     if (x > half) x -= M;
     return x;
 }
 
+// The two residues (elements i and i + 1) of built-in modulus T as one word; 0 where T takes no part.
+template <int T>
+__device__ __forceinline__ void crt_load(const CrtParams& p, const short* __restrict__ res, long long i, bool vec,
+                                         bool two, unsigned int (&word)[kNumWideModuli]) {
+    word[T] = 0;
+    if (p.mask >> T & 1u) {
+        const short* src = res + p.offset[T] + i;
+        if (vec) {
+            word[T] = __ldg(reinterpret_cast<const unsigned int*>(src));
+        } else {
+            word[T] = (unsigned short)src[0];
+            if (two) word[T] |= (unsigned int)(unsigned short)src[1] << 16;
+        }
+    }
+    if constexpr (T + 1 < kNumWideModuli) crt_load<T + 1>(p, res, i, vec, two, word);
+}
+
+template <int T>
+__device__ __forceinline__ void crt_accumulate(const CrtParams& p, const unsigned int (&word)[kNumWideModuli],
+                                               long long (&a)[2][4]) {
+    if (p.mask >> T & 1u) {
+        const int r0 = (int)(word[T] << 16) >> 16, r1 = (int)word[T] >> 16;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            a[0][k] += (long long)r0 * (long long)p.w[T][k];
+            a[1][k] += (long long)r1 * (long long)p.w[T][k];
+        }
+    }
+    if constexpr (T + 1 < kNumWideModuli) crt_accumulate<T + 1>(p, word, a);
+}
+
 // A thread takes two neighbouring elements: one 4-byte load per modulus (a warp reads whole 128-byte
-// lines), all loads of a batch of kCrtBatch moduli in flight together (with one 2-byte load at a time
-// the kernel was bound by load latency), and the two 128-bit results leave as one 32-byte sector.
+// lines), the loads of all moduli in flight together, the loop over the moduli unrolled at compile time
+// (the limbs of W_T are then operands straight from the parameter bank), and the two 128-bit results
+// leave as one 32-byte sector.
 __global__ void __launch_bounds__(256)
 wide_crt_kernel(const short* __restrict__ res, long long count, const __grid_constant__ CrtParams p,
-                long long* __restrict__ out) {
+                long long* __restrict__ out, int vec_ok) {
     const i128 M = (i128)(((u128)p.M_hi << 64) | p.M_lo);
     const i128 half = (i128)(((u128)p.half_hi << 64) | p.half_lo);
     const long long pairs = (count + 1) / 2;
-    // every modulus' array starts on a 4-byte boundary
-    const bool vec = (count & 1) == 0 && (reinterpret_cast<uintptr_t>(res) & 3) == 0;
     for (long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x; g < pairs;
          g += (long long)gridDim.x * blockDim.x) {
         const long long i = 2 * g;
         const bool two = i + 1 < count;
-        unsigned long long a[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
-        for (int t0 = 0; t0 < p.n; t0 += kCrtBatch) {
-            unsigned int word[kCrtBatch];
-#pragma unroll
-            for (int u = 0; u < kCrtBatch; ++u) {
-                word[u] = 0;
-                if (t0 + u < p.n) {
-                    const short* src = res + (long long)(t0 + u) * count + i;
-                    if (vec) {
-                        word[u] = __ldg(reinterpret_cast<const unsigned int*>(src));
-                    } else {
-                        word[u] = (unsigned short)src[0];
-                        if (two) word[u] |= (unsigned int)(unsigned short)src[1] << 16;
-                    }
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < kCrtBatch; ++u) {
-                if (t0 + u >= p.n) break;
-                const int m = p.m[t0 + u];
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    int r = (int)(short)(word[u] >> (16 * e));
-                    r += r < 0 ? m : 0;
-                    const unsigned int ru = (unsigned int)r;
-                    a[e][0] += (unsigned long long)ru * p.w[t0 + u][0];
-                    a[e][1] += (unsigned long long)ru * p.w[t0 + u][1];
-                    a[e][2] += (unsigned long long)ru * p.w[t0 + u][2];
-                    a[e][3] += (unsigned long long)ru * p.w[t0 + u][3];
-                }
-            }
-        }
-        const i128 x0 = crt_reduce(a[0][0], a[0][1], a[0][2], a[0][3], p, M, half);
+        unsigned int word[kNumWideModuli];
+        crt_load<0>(p, res, i, vec_ok != 0, two, word);
+        long long a[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+        crt_accumulate<0>(p, word, a);
+        const i128 x0 = crt_reduce(a[0], p, M, half);
         longlong2* dst = reinterpret_cast<longlong2*>(out + 2 * i);
         dst[0] = make_longlong2((long long)(unsigned long long)(u128)x0, (long long)(x0 >> 64));
         if (two) {
-            const i128 x1 = crt_reduce(a[1][0], a[1][1], a[1][2], a[1][3], p, M, half);
+            const i128 x1 = crt_reduce(a[1], p, M, half);
             dst[1] = make_longlong2((long long)(unsigned long long)(u128)x1, (long long)(x1 >> 64));
         }
     }
 }
 
-bool build_crt_params(const int* moduli, int n, CrtParams* c) {
-    c->n = n;
+// moduli[t] (each one of the built-in set, no repeats) with its residues at res + t * count.
+bool build_crt_params(const int* moduli, int n, long long count, CrtParams* c) {
     u128 M = 1;
     for (int t = 0; t < n; ++t) M *= (u128)moduli[t];
     for (int t = 0; t < n; ++t) {
         const int m = moduli[t];
+        int T = 0;
+        while (T < kNumWideModuli && kWideModuli[T] != m) ++T;
+        if (T == kNumWideModuli || (c->mask >> T & 1u)) return false;
         const u128 Mt = M / (u128)m;
         const int mt_mod = (int)(Mt % (u128)m);
         int inv = 0;
@@ -215,15 +237,16 @@ bool build_crt_params(const int* moduli, int n, CrtParams* c) {
             if ((mt_mod * a) % m == 1) inv = a;
         if (!inv) return false;
         const u128 W = Mt * (u128)inv;  // < M
-        c->m[t] = m;
-        for (int k = 0; k < 4; ++k) c->w[t][k] = (unsigned int)(W >> (32 * k));
+        c->mask |= 1u << T;
+        c->offset[T] = (long long)t * count;
+        for (int k = 0; k < 4; ++k) c->w[T][k] = (int)((W >> (31 * k)) & 0x7FFFFFFFu);
     }
-    for (int k = 0; k < 4; ++k) c->M[k] = (unsigned int)(M >> (32 * k));
+    for (int k = 0; k < 4; ++k) c->M[k] = (int)((M >> (31 * k)) & 0x7FFFFFFFu);
     c->M_lo = (unsigned long long)M;
     c->M_hi = (unsigned long long)(M >> 64);
     c->half_lo = (unsigned long long)(M / 2);
     c->half_hi = (unsigned long long)((M / 2) >> 64);
-    c->M_as_double = (double)c->M_hi * 18446744073709551616.0 + (double)c->M_lo;
+    c->inv_M = 1.0 / ((double)c->M_hi * 18446744073709551616.0 + (double)c->M_lo);
     return true;
 }
 
@@ -315,21 +338,19 @@ static awe_status_t launch_residues(awe_handle_t h, const int64_t* X_dev, int64_
                                     int8_t* res_dev, void* stream) {
     if (!h || !X_dev || !res_dev || count <= 0) return AWE_ERR_INVALID_ARG;
     if ((uintptr_t)X_dev % 16 || (uintptr_t)res_dev % 4) return AWE_ERR_ALIGNMENT;
+    // residues of moduli[t] go to res_dev + t * count; every modulus must be one of the built-in set
     ResidueParams p = {};
-    p.n = n;
     for (int t = 0; t < n; ++t) {
-        const unsigned int m = (unsigned int)moduli[t];
-        p.mf[t] = (float)m;
-        p.inv_m[t] = 1.0f / (float)m;
-        p.c1f[t] = (float)((1u << 14) % m);
-        p.c2f[t] = (float)((1u << 28) % m);
-        p.c3f[t] = (float)((1ull << 42) % m);
-        p.lo[t] = -(float)(m / 2);
-        p.hi[t] = (float)((m + 1) / 2) - 1.0f;
+        int T = 0;
+        while (T < kNumWideModuli && kWideModuli[T] != moduli[t]) ++T;
+        if (T == kNumWideModuli || (p.mask >> T & 1u)) return AWE_ERR_UNSUPPORTED;
+        p.mask |= 1u << T;
+        p.offset[T] = (long long)t * count;
     }
-    const long long groups = (count + 3) / 4;
+    const long long groups = (count + kResPerThread - 1) / kResPerThread;
     const unsigned blocks = (unsigned)std::min<long long>((groups + 255) / 256, (long long)h->sm_count * 16);
-    wide_residues_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const long long*)X_dev, count, p, res_dev);
+    const int vec = (count % 8 == 0) && ((uintptr_t)res_dev % 8 == 0);
+    wide_residues_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const long long*)X_dev, count, p, res_dev, vec);
     if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
     h->launches += 1;
     return AWE_OK;
@@ -345,9 +366,12 @@ static awe_status_t launch_crt(awe_handle_t h, const int16_t* res_dev, int64_t c
     if (!h || !res_dev || !out_dev || count <= 0) return AWE_ERR_INVALID_ARG;
     if ((uintptr_t)res_dev % 2 || (uintptr_t)out_dev % 16) return AWE_ERR_ALIGNMENT;
     CrtParams c = {};
-    if (!build_crt_params(moduli, n, &c)) return AWE_ERR_UNSUPPORTED;
+    if (!build_crt_params(moduli, n, count, &c)) return AWE_ERR_UNSUPPORTED;
     const unsigned blocks = (unsigned)std::min<long long>(((count + 1) / 2 + 255) / 256, (long long)h->sm_count * 16);
-    wide_crt_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const short*)res_dev, count, c, (long long*)out_dev);
+    // every modulus' array starts on a 4-byte boundary
+    const int vec_ok = (count & 1) == 0 && ((uintptr_t)res_dev & 3) == 0;
+    wide_crt_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const short*)res_dev, count, c, (long long*)out_dev,
+                                                             vec_ok);
     if (cudaGetLastError() != cudaSuccess) return AWE_ERR_CUDA;
     h->launches += 1;
     return AWE_OK;

@@ -62,6 +62,38 @@ def test_crt_kernel():
     got = _to_python_ints(out.cpu().numpy())
     assert [int(g) for g in got] == xs
     assert [rns.crt_symmetric(res[:, i], rns.RNS_SET_FP64) for i in range(20)] == xs[:20]
+    # an even count takes the path with one 4-byte load per modulus and pair of elements
+    assert len(xs) % 2 == 1
+    even = torch.empty((len(xs) - 1, 2), dtype=torch.int64, device="cuda")
+    b.awe_wide_crt(h, torch.from_numpy(np.ascontiguousarray(res[:, :-1])).cuda(), len(xs) - 1, even)
+    assert [int(g) for g in _to_python_ints(even.cpu().numpy())] == xs[:-1]
+    # other representatives of the same residue classes give the same integers
+    # (|r| < m: the non-negative one, or that minus m)
+    shifted = np.array([[x % m - (m if (i + m) % 3 == 0 and x % m else 0) for i, x in enumerate(xs)]
+                        for m in rns.RNS_SET_FP64], dtype=np.int16)
+    assert (np.abs(shifted) < np.array(rns.RNS_SET_FP64)[:, None]).all() and (shifted < 0).any()
+    b.awe_wide_crt(h, torch.from_numpy(shifted).cuda(), len(xs), out)
+    assert [int(g) for g in _to_python_ints(out.cpu().numpy())] == xs
+
+
+def test_residues_of_values_on_the_rounding_boundaries():
+    """x = q m + r for every symmetric residue r of every modulus, at small and at 53-bit magnitudes and
+    both signs: covers the ties of the even modulus and the ends of every range."""
+    h = gu.handle()
+    xs = []
+    for m in rns.RNS_SET_FP64:
+        for r in range(-(m // 2), (m + 1) // 2):
+            for q in (0, 1, -1, 3, (B53 // m) - 2, -((B53 // m) - 2), 2 ** 40 + 1, -(2 ** 40) - 5):
+                xs.append(q * m + r)
+    X = np.array(xs, dtype=np.int64)
+    assert np.abs(X).max() <= B53
+    res = torch.empty((len(rns.RNS_SET_FP64), len(xs)), dtype=torch.int8, device="cuda")
+    b.awe_wide_residues(h, torch.from_numpy(X).cuda(), len(xs), res)
+    got = res.cpu().numpy()
+    for t, m in enumerate(rns.RNS_SET_FP64):
+        lo = -(m // 2)
+        want = ((X.astype(object) - lo) % m + lo).astype(np.int8)
+        assert np.array_equal(got[t], want), m
 
 
 @pytest.mark.parametrize("shape", [(1, 1, 1), (60, 40, 200), (130, 270, 513)])
