@@ -190,6 +190,27 @@ def test_forced_k_segments_worst_case_inputs(k_chunk):
         assert np.array_equal(got, want)
 
 
+@pytest.mark.parametrize("K", [116480, 232960])
+def test_planes_of_extreme_values_at_and_beyond_k_star(K):
+    """Section 3.4 through awe_gemm_planes: every stored plane value +-12 (the width-12 record, c = 12,
+    K* = 116,508).  K = 116,480 fits one segment with |P| = 144 K just below 2^24; K = 232,960 must be
+    cut.  Closed form: every product is +-144 K, so C = +-144 K (sum of the coefficients) / D."""
+    enc = b.ENC_FP16SIG_AWE12
+    d = b.awe_encoding_info(enc)
+    assert d.c_a == 12 and d.c_b == 12 and d.k_star == 116508 and (K <= d.k_star) == (K == 116480)
+    M, N = 40, 72
+    pa = np.full((d.n_planes_a, M, K), 12, dtype=np.int8)
+    pb = np.full((d.n_planes_b, N, K), 12, dtype=np.int8)
+    pb[:, 1::2] = -12
+    packed_a = gu.padded_planes(np.stack([pl.pack_e2m1(x) for x in pa]), K)
+    packed_b = gu.padded_planes(np.stack([pl.pack_e2m1(x) for x in pb]), K)
+    got = gu.gpu_gemm_planes(packed_a, packed_b, M, N, K, enc, b.C_I64)
+    total = sum(int(l) for l in d.ell[:d.r]) * 144 * K
+    assert total % (1 << d.log2D) == 0
+    want = total >> d.log2D
+    assert np.all(got[:, 0::2] == want) and np.all(got[:, 1::2] == -want)
+
+
 def test_int64_output_beyond_32_bits():
     """K = 2^18 with all entries -128: C = 2^14 K = 2^32, needs the 64-bit path."""
     M, N, K = 128, 256, 1 << 18
