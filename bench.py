@@ -373,7 +373,8 @@ def main():
     def want(name):
         return args.context == "all" or name in args.context.split(",")
 
-    if rank == 0 and not args.no_extras:
+    # the context measurements are single-GPU work: in a multi-GPU run every rank finishes at the same time
+    if rank == 0 and world == 1 and not args.no_extras:
         ctx = {}
         if want("base13"):
             # prior-work 9-GEMM base-13 scheme through the same kernels, same inputs
