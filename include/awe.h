@@ -285,7 +285,8 @@ awe_status_t awe_gemm_exact_wide(awe_handle_t h, const int64_t* A_dev, const int
  *   - The first call on a device looks up the array's device address and the device's properties,
  *     clears the status word and (once per process) page-locks a small host mirror of the status words
  *     in place; the first use of an encoding on a device uploads its tables and waits for that copy
- *     (room for 96 tables per device).  Make those first calls before any stream capture.
+ *     (room for 96 tables per device).  These first calls synchronise `stream`, which a stream that is
+ *     being captured does not allow.
  *   - Every call on a device shares the one array, which keeps the previous call's planes: calls
  *     whose kernels could overlap on the GPU (different streams, or several host threads) race
  *     and must be serialised by the caller.  Nothing in it needs to start at zero except the status
