@@ -192,7 +192,7 @@ def main():
                     help="INT8xINT8 record of the timed step (the headline metric is awe6)")
     ap.add_argument("--no-extras", action="store_true", help="skip the context measurements")
     ap.add_argument("--context", default="all",
-                    help="comma list of context measurements to run: base13, mixed, derived, int8, configs, ceiling, "
+                    help="comma list of context measurements to run: sustained, base13, mixed, derived, int8, configs, ceiling, "
                          "reconstruct (default: all)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     args = ap.parse_args()
@@ -376,6 +376,22 @@ def main():
     # the context measurements are single-GPU work: in a multi-GPU run every rank finishes at the same time
     if rank == 0 and world == 1 and not args.no_extras:
         ctx = {}
+        if want("sustained"):
+            # the same step 300 times back to back (about 0.4 s): long enough for the power regulator to settle,
+            # reported beside the burst figure of the timed region above
+            for _ in range(3):
+                step()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(300):
+                step()
+            e1.record()
+            torch.cuda.synchronize()
+            ms300 = e0.elapsed_time(e1) / 300
+            ctx["sustained_300_steps"] = {"TOPS": ops / (ms300 * 1e-3) / 1e12, "ms_per_step": ms300,
+                                          "sm_mhz_in_gemm_kernel": b.awe_last_gemm_clock_mhz(h)}
+            time.sleep(1.0)  # let the part cool before the next short measurement
         if want("base13"):
             # prior-work 9-GEMM base-13 scheme through the same kernels, same inputs
             enc9 = b.ENC_INT8_BASE13_9
